@@ -1,0 +1,130 @@
+/*
+ * libmate -- multi-view (row head / column head / global prefix) sparse self-attention for
+ * flattened tables, hand-written CUDA for sm_100a.
+ *
+ * The operation is the one defined in Section 3 of "MATE: Multi-view Attention for Table
+ * Transformer Efficiency": for head i and token position k the output is a softmax-weighted sum of
+ * the values of the positions in the attention pattern A^i_k,
+ *     k in Q (the query/text prefix)  ->  A = every position (except padding)
+ *     row head,    k not in Q         ->  A = Q  u  { j : r_j = r_k }
+ *     column head, k not in Q         ->  A = Q  u  { j : c_j = c_k }
+ * applied after the Q/K/V projections (Q, K, V are inputs here).  Section 3.1's observation that
+ * every head may traverse the tokens in its own data-dependent, deterministic order is what
+ * mate_plan pre-computes: in a head's view order each table token's keys are one contiguous
+ * segment plus the prefix block.
+ *
+ * Conventions (the paper leaves them open):
+ *   - Q is the first prefix_len positions; their row and column ids must be 0.
+ *   - a negative id marks padding (both arrays must agree).  Padding keys are never attended;
+ *     padding query rows return O = 0, LSE = -inf and zero gradients; values stored at padding
+ *     positions are ignored.
+ *   - a table token whose id is 0 is an ordinary table token (segment 0).
+ *   - masking removes a key from the softmax support; `scale` multiplies q.k before the softmax.
+ *   - LSE is the natural-log logsumexp of the scaled scores over A.
+ *
+ * All tensor pointers are DEVICE pointers unless a comment says "host".  The library never keeps
+ * or frees caller memory.  Every call returns a status (0 = MATE_OK, negative = error); nothing
+ * throws across this boundary.  Calls taking a `stream` (a cudaStream_t passed as void*) enqueue
+ * work on it and return without waiting, except mate_plan, which waits for its own kernels.
+ */
+#ifndef MATE_H_
+#define MATE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mate_plan_s mate_plan_t;
+
+enum {
+    MATE_OK = 0,
+    MATE_ERR_INVALID_ARG = -1, /* null pointer, bad size, ids that break the conventions above     */
+    MATE_ERR_UNSUPPORTED = -2, /* head dim / dtype / implementation not available for these sizes   */
+    MATE_ERR_ALIGNMENT = -3,   /* a tensor pointer is not 16-byte aligned                           */
+    MATE_ERR_CUDA = -4,        /* a CUDA runtime call failed (the CUDA error is left in place)      */
+    MATE_ERR_TIMEOUT = -5,     /* a bounded wait inside a kernel expired (see mate_plan_status)     */
+    MATE_ERR_NOMEM = -6,       /* host or device allocation failed                                  */
+    MATE_ERR_WORKSPACE = -7    /* workspace pointer null or smaller than mate_attn_workspace_bytes  */
+};
+
+enum { MATE_BF16 = 0, MATE_F32 = 1 };          /* element type of Q, K, V, O, dO, dQ, dK, dV */
+enum { MATE_VIEW_ROW = 0, MATE_VIEW_COL = 1 }; /* entries of head_view                      */
+
+/* flags for mate_attn_fwd / mate_attn_bwd: which implementation runs.
+ *   AUTO     tensor-core (tcgen05) kernels when dtype = bf16 and d = 64, otherwise the SIMT kernels
+ *   SIMT     one-warp-per-row fp32-arithmetic kernels (any dtype, d <= 128): the debug path
+ *   TCGEN05  tensor-core kernels or MATE_ERR_UNSUPPORTED */
+enum { MATE_IMPL_AUTO = 0, MATE_IMPL_SIMT = 1, MATE_IMPL_TCGEN05 = 2 };
+
+const char *mate_status_string(int status);
+
+/* Pre-computes, for both views, the per-head token order of Section 3.1 (Figure 2): a stable
+ * counting sort of the positions by (prefix, table id, padding), i.e. the row-order / column-order
+ * traversal of the table, together with the segment offsets and the tile work-lists the attention
+ * kernels walk.  Integer work; the result is unique (ties keep the original order).
+ *
+ *   row_ids, col_ids  device int32 [B, N]
+ *   prefix_len        |Q|, 0 <= prefix_len <= N
+ *   head_view         HOST uint8 [H], MATE_VIEW_ROW or MATE_VIEW_COL per head (any mix, one view
+ *                     may have no head)
+ *   max_row_id, max_col_id   inclusive upper bounds of the non-negative ids
+ *   out               receives a plan owned by the library; free it with mate_plan_destroy
+ *
+ * The plan can be reused for any number of forward/backward calls, layers and head dims.  Runs its
+ * kernels on `stream` and waits for them (it allocates device memory, so call it outside a stream
+ * capture).  Ids that break the conventions give MATE_ERR_INVALID_ARG and no plan. */
+int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len,
+              const uint8_t *head_view, int H, int max_row_id, int max_col_id, void *stream,
+              mate_plan_t **out);
+
+/* Copies one view's order to HOST arrays (any pointer may be null to skip it):
+ *   perm      int32 [B, N]          perm[b][t] = original position of the t-th token of the view
+ *   inv_perm  int32 [B, N]          inverse of perm
+ *   seg_off   int32 [B, max_id+2]   tokens with id s occupy view positions [seg_off[s], seg_off[s+1]);
+ *                                   seg_off[0] = prefix_len, seg_off[max_id+1] = number of
+ *                                   non-padding tokens */
+int mate_plan_get(const mate_plan_t *plan, int view, int32_t *perm, int32_t *inv_perm,
+                  int32_t *seg_off);
+
+/* Number of unmasked (query, key) pairs per example and head (the O(ng + nb) count of Table 1):
+ * HOST int64 [B, H].  Forward work is 4*d flops per pair, backward 10*d. */
+int mate_plan_useful_pairs(const mate_plan_t *plan, int64_t *pairs);
+
+/* Waits for `stream` and returns MATE_ERR_TIMEOUT if any kernel that used this plan gave up on a
+ * bounded wait since the last call (its outputs are then undefined), MATE_ERR_CUDA if the stream
+ * reports an error, else MATE_OK. */
+int mate_plan_status(const mate_plan_t *plan, void *stream);
+
+int mate_plan_destroy(mate_plan_t *plan);
+
+/* Scratch sizes (bytes) the caller must provide to mate_attn_fwd / mate_attn_bwd for head dim d,
+ * element type dtype and implementation `flags`.  Either size may be 0. */
+int mate_attn_workspace_bytes(const mate_plan_t *plan, int d, int dtype, unsigned flags,
+                              size_t *fwd_bytes, size_t *bwd_bytes);
+
+/* Forward: the head formula of Section 3 for every (b, h, k).
+ *   Q, K, V   [B, H, N, d] contiguous, dtype elements, 16-byte aligned
+ *   O         [B, H, N, d] same type, fully overwritten, original token order
+ *   LSE       float32 [B, H, N]
+ *   workspace device scratch of at least fwd_bytes (may be null when that is 0), 256-byte aligned;
+ *             contents are undefined afterwards; concurrent calls need separate workspaces
+ * d must be a multiple of 8 and at most 128.  Asynchronous on `stream`. */
+int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d,
+                  int dtype, float scale, void *O, float *LSE, void *workspace,
+                  size_t workspace_bytes, unsigned flags, void *stream);
+
+/* Backward of mate_attn_fwd (derived from the Section 3 head formula; the paper states no
+ * backward): given O and LSE of the forward call and dO, writes dQ, dK, dV (fully overwritten,
+ * no accumulation into previous contents).  Same layouts, types and rules as the forward. */
+int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
+                  const void *O, const float *LSE, const void *dO, int d, int dtype, float scale,
+                  void *dQ, void *dK, void *dV, void *workspace, size_t workspace_bytes,
+                  unsigned flags, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MATE_H_ */

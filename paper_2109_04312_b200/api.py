@@ -1,0 +1,209 @@
+"""ctypes binding of libmate.so (same names as the C entry points; marshalling only)."""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libmate.so")
+
+IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+VIEW_ROW, VIEW_COL = 0, 1
+_BF16, _F32 = 0, 1
+
+_lib = None
+
+
+class MateError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (where, _status_string(status), status))
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    """Loads the CUDA library; there is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            "libmate.so is not built: run `python -m paper_2109_04312_b200.build` "
+            "(needs nvcc); there is no CPU or PyTorch fallback")
+    lib = C.CDLL(_LIB_PATH)
+    vp, i32, u32, f32, sz = C.c_void_p, C.c_int, C.c_uint, C.c_float, C.c_size_t
+    lib.mate_status_string.restype = C.c_char_p
+    lib.mate_status_string.argtypes = [i32]
+    lib.mate_plan.restype = i32
+    lib.mate_plan.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, vp, C.POINTER(vp)]
+    lib.mate_plan_get.restype = i32
+    lib.mate_plan_get.argtypes = [vp, i32, vp, vp, vp]
+    lib.mate_plan_useful_pairs.restype = i32
+    lib.mate_plan_useful_pairs.argtypes = [vp, vp]
+    lib.mate_plan_status.restype = i32
+    lib.mate_plan_status.argtypes = [vp, vp]
+    lib.mate_plan_destroy.restype = i32
+    lib.mate_plan_destroy.argtypes = [vp]
+    lib.mate_attn_workspace_bytes.restype = i32
+    lib.mate_attn_workspace_bytes.argtypes = [vp, i32, i32, u32, C.POINTER(sz), C.POINTER(sz)]
+    lib.mate_attn_fwd.restype = i32
+    lib.mate_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, sz, u32, vp]
+    lib.mate_attn_bwd.restype = i32
+    lib.mate_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, vp, sz, u32, vp]
+    _lib = lib
+    return lib
+
+
+def _status_string(status):
+    try:
+        return _load().mate_status_string(status).decode()
+    except Exception:
+        return "?"
+
+
+def _check(status, where):
+    if status != 0:
+        raise MateError(status, where)
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t):
+    if t.dtype == torch.bfloat16:
+        return _BF16
+    if t.dtype == torch.float32:
+        return _F32
+    raise TypeError("libmate takes bfloat16 or float32 tensors, got %s" % t.dtype)
+
+
+def _dev(t, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise ValueError("%s must be a contiguous CUDA tensor" % name)
+    return C.c_void_p(t.data_ptr())
+
+
+class Plan:
+    """Owner of a mate_plan_t*: the pre-computed per-view order (see mate_plan)."""
+
+    def __init__(self, handle, B, N, P, H, max_row_id, max_col_id, device):
+        self._h = handle
+        self.B, self.N, self.P, self.H = B, N, P, H
+        self.max_id = (max_row_id, max_col_id)
+        self.device = device
+        self._ws = {}
+
+    def get(self, view):
+        """(perm, inv_perm, seg_off) of one view as numpy int32 arrays."""
+        perm = np.empty((self.B, self.N), np.int32)
+        inv = np.empty((self.B, self.N), np.int32)
+        seg = np.empty((self.B, self.max_id[view] + 2), np.int32)
+        _check(_load().mate_plan_get(self._h, view, perm.ctypes.data, inv.ctypes.data, seg.ctypes.data),
+               "mate_plan_get")
+        return perm, inv, seg
+
+    def useful_pairs(self):
+        out = np.empty((self.B, self.H), np.int64)
+        _check(_load().mate_plan_useful_pairs(self._h, out.ctypes.data), "mate_plan_useful_pairs")
+        return out
+
+    def status(self):
+        _check(_load().mate_plan_status(self._h, _stream()), "mate_plan_status")
+
+    def destroy(self):
+        if self._h is not None:
+            _load().mate_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_id=None) -> Plan:
+    """row_ids, col_ids: int32 CUDA tensors [B, N]; head_view: sequence of 0 (row) / 1 (column)."""
+    if row_ids.dtype != torch.int32 or col_ids.dtype != torch.int32 or row_ids.shape != col_ids.shape \
+            or row_ids.dim() != 2:
+        raise ValueError("row_ids / col_ids must be int32 tensors of the same [B, N] shape")
+    B, N = row_ids.shape
+    hv = np.ascontiguousarray(np.asarray(head_view, dtype=np.uint8))
+    if max_row_id is None:
+        max_row_id = max(int(row_ids.max().item()), 0)
+    if max_col_id is None:
+        max_col_id = max(int(col_ids.max().item()), 0)
+    handle = C.c_void_p()
+    with torch.cuda.device(row_ids.device):
+        _check(_load().mate_plan(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N,
+                                 int(prefix_len), hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
+                                 int(max_col_id), _stream(), C.byref(handle)), "mate_plan")
+    return Plan(handle, B, N, int(prefix_len), int(hv.shape[0]), int(max_row_id), int(max_col_id),
+                row_ids.device)
+
+
+def mate_attn_workspace_bytes(plan, d, dtype, impl=IMPL_AUTO):
+    f, b = C.c_size_t(0), C.c_size_t(0)
+    _check(_load().mate_attn_workspace_bytes(plan._h, int(d), dtype, impl, C.byref(f), C.byref(b)),
+           "mate_attn_workspace_bytes")
+    return f.value, b.value
+
+
+def _workspace(plan, nbytes, key):
+    if nbytes == 0:
+        return None
+    ws = plan._ws.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device=plan.device)
+        plan._ws[key] = ws
+    return ws
+
+
+def mate_attn_fwd(plan, Q, K, V, scale=None, impl=IMPL_AUTO, out=None, lse=None, workspace=None):
+    """Q, K, V: [B, H, N, d] CUDA tensors (bf16 or f32).  Returns (O, LSE) in original token order."""
+    B, H, N, d = Q.shape
+    if (B, H, N) != (plan.B, plan.H, plan.N) or K.shape != Q.shape or V.shape != Q.shape:
+        raise ValueError("tensor shapes do not match the plan")
+    dt = _dtype_code(Q)
+    if scale is None:
+        scale = 1.0 / float(d) ** 0.5
+    O = torch.empty_like(Q) if out is None else out
+    LSE = torch.empty((B, H, N), dtype=torch.float32, device=Q.device) if lse is None else lse
+    need, _ = mate_attn_workspace_bytes(plan, d, dt, impl)
+    ws = workspace if workspace is not None else _workspace(plan, need, "fwd")
+    with torch.cuda.device(Q.device):
+        _check(_load().mate_attn_fwd(plan._h, _dev(Q, "Q"), _dev(K, "K"), _dev(V, "V"), d, dt,
+                                     float(scale), _dev(O, "O"), _dev(LSE, "LSE"),
+                                     C.c_void_p(ws.data_ptr()) if ws is not None else None,
+                                     ws.numel() if ws is not None else 0, impl, _stream()),
+               "mate_attn_fwd")
+    return O, LSE
+
+
+def mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale=None, impl=IMPL_AUTO, workspace=None):
+    """Returns (dQ, dK, dV)."""
+    B, H, N, d = Q.shape
+    if (B, H, N) != (plan.B, plan.H, plan.N):
+        raise ValueError("tensor shapes do not match the plan")
+    for t in (K, V, O, dO):
+        if t.shape != Q.shape or t.dtype != Q.dtype:
+            raise ValueError("K, V, O, dO must match Q in shape and dtype")
+    dt = _dtype_code(Q)
+    if scale is None:
+        scale = 1.0 / float(d) ** 0.5
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(Q), torch.empty_like(Q)
+    _, need = mate_attn_workspace_bytes(plan, d, dt, impl)
+    ws = workspace if workspace is not None else _workspace(plan, need, "bwd")
+    with torch.cuda.device(Q.device):
+        _check(_load().mate_attn_bwd(plan._h, _dev(Q, "Q"), _dev(K, "K"), _dev(V, "V"), _dev(O, "O"),
+                                     _dev(LSE, "LSE"), _dev(dO, "dO"), d, dt, float(scale),
+                                     _dev(dQ, "dQ"), _dev(dK, "dK"), _dev(dV, "dV"),
+                                     C.c_void_p(ws.data_ptr()) if ws is not None else None,
+                                     ws.numel() if ws is not None else 0, impl, _stream()),
+               "mate_attn_bwd")
+    return dQ, dK, dV

@@ -1,0 +1,149 @@
+// Per-view token order (Section 3.1: every head traverses the table in its own row-order or
+// column-order, "data-dependent but deterministic"): a stable counting sort of the positions by
+// (prefix, table id, padding).  One CTA per (example, view); integer work only.
+#include "mate_internal.h"
+
+namespace mate {
+
+namespace {
+
+constexpr int kPlanThreads = 1024;
+constexpr int kSmemIds = 4096;  // id histograms up to this many entries live in shared memory
+
+__device__ __forceinline__ int warp_inclusive_scan(int v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+    }
+    return v;
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N, int P,
+            ViewPlan rowv, ViewPlan colv, int32_t *__restrict__ n_valid_out,
+            int32_t *__restrict__ status) {
+    __shared__ int32_t s_cursor[kSmemIds];
+    __shared__ int s_n_valid;
+
+    const int b = blockIdx.x, view = blockIdx.y;
+    const ViewPlan &vp = view ? colv : rowv;
+    const int32_t *ids = (view ? col_ids : row_ids) + (size_t)b * N;
+    const int32_t *oth = (view ? row_ids : col_ids) + (size_t)b * N;
+    const int S = vp.max_id + 2;
+    int32_t *seg_off = vp.seg_off + (size_t)b * S;
+    int32_t *perm = vp.perm + (size_t)b * N;
+    int32_t *inv_perm = vp.inv_perm + (size_t)b * N;
+    volatile int32_t *cur = (S <= kSmemIds) ? s_cursor : (vp.cursor + (size_t)b * S);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    for (int i = tid; i < S; i += kPlanThreads) cur[i] = 0;
+    __syncthreads();
+
+    // A position is a table token iff it lies behind the prefix and both ids are valid; anything
+    // else behind the prefix is treated as padding so that every later index stays in range even
+    // when the input breaks the conventions (which is reported through `status`).
+    auto is_table = [&](int k) {
+        int id = ids[k];
+        return k >= P && id >= 0 && id <= vp.max_id && oth[k] >= 0;
+    };
+
+    // 1. validate + histogram of table ids
+    bool bad = false;
+    for (int k = tid; k < N; k += kPlanThreads) {
+        int id = ids[k], o = oth[k];
+        if (k < P) {
+            bad |= (id != 0) | (o != 0);
+        } else if (id < 0) {
+            bad |= (o >= 0);
+        } else if (o < 0 || id > vp.max_id) {
+            bad = true;
+        } else {
+            atomicAdd((int *)&cur[id], 1);
+        }
+    }
+    if (bad) atomicOr(status, 1);
+    __syncthreads();
+
+    // 2. exclusive scan of the histogram -> segment offsets (warp 0, 32 entries per step)
+    if (warp == 0) {
+        int carry = P;
+        for (int base = 0; base < S; base += 32) {
+            int i = base + lane;
+            int c = (i < S - 1) ? cur[i] : 0;
+            int incl = warp_inclusive_scan(c, lane);
+            int excl = carry + incl - c;
+            if (i < S) {
+                seg_off[i] = excl;
+                cur[i] = excl;
+            }
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (lane == 0) {
+            s_n_valid = carry;
+            if (view == 0) n_valid_out[b] = carry;
+        }
+    }
+    __syncthreads();
+    const int n_valid = s_n_valid;
+
+    // 3. stable scatter (warp 0 walks the positions in order, 32 at a time; lanes holding the same
+    //    id are ranked by lane, so equal ids keep their original order)
+    if (warp == 0) {
+        int pad_cursor = n_valid;
+        for (int base = 0; base < N; base += 32) {
+            int k = base + lane;
+            bool in = k < N;
+            bool table = in && is_table(k);
+            bool padding = in && !table && k >= P;
+            int id = table ? ids[k] : 0;
+            int key = table ? id : (padding ? -1 : (int)0x80000000 + lane);
+            unsigned grp = __match_any_sync(0xffffffffu, key);
+            int rank = __popc(grp & ((1u << lane) - 1u));
+            int cnt = __popc(grp);
+            int basep = 0;
+            if (table) basep = cur[id];
+            __syncwarp();
+            if (table && rank == 0) cur[id] = basep + cnt;
+            __syncwarp();
+            int n_pad = __popc(__ballot_sync(0xffffffffu, padding));
+            int pos = k;  // prefix tokens keep their positions
+            if (table) pos = basep + rank;
+            if (padding) pos = pad_cursor + rank;
+            pad_cursor += n_pad;
+            if (in) {
+                perm[pos] = k;
+                inv_perm[k] = pos;
+            }
+        }
+    }
+    __syncthreads();
+
+    // 4. per view position: the key range of its own segment
+    int32_t *seg_lo = vp.seg_lo + (size_t)b * N, *seg_hi = vp.seg_hi + (size_t)b * N;
+    for (int t = tid; t < N; t += kPlanThreads) {
+        int lo = 0, hi = 0;
+        if (t < P) {
+            hi = n_valid;
+        } else if (t < n_valid) {
+            int id = ids[perm[t]];
+            lo = seg_off[id];
+            hi = seg_off[id + 1];
+        }
+        seg_lo[t] = lo;
+        seg_hi[t] = hi;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P,
+                                const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
+                                int32_t *status, cudaStream_t stream) {
+    dim3 grid(B, 2);
+    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, P, rowv, colv, n_valid,
+                                                   status);
+    return cudaGetLastError();
+}
+
+}  // namespace mate

@@ -1,0 +1,288 @@
+// SIMT (no tensor core) kernels: one warp per query row (forward, dQ) or per key row (dK/dV).
+// fp32 arithmetic whatever the storage type; this is the debug / any-head-dim path and the
+// reference the tensor-core kernels were brought up against on the device.
+//
+// In a head's view order (see mate_plan) the keys of query row t are
+//     [0, P)  u  [max(seg_lo[t], P), seg_hi[t])
+// which is the attention pattern A of Section 3 for both table rows (own segment plus prefix) and
+// prefix rows (seg_lo = 0, seg_hi = n_valid).  The pattern is symmetric, so the queries that
+// attend to key t are the same two ranges; dK/dV therefore need no atomics.
+#include <cuda_bf16.h>
+
+#include "mate_internal.h"
+
+namespace mate {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 4;
+constexpr int kMaxD = 128;
+constexpr int kAccPerLane = kMaxD / 32;
+
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void from_f(float &dst, float x) { dst = x; }
+__device__ __forceinline__ void from_f(__nv_bfloat16 &dst, float x) { dst = __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <typename T>
+__device__ __forceinline__ float dot_row(const float *__restrict__ a_smem, const T *__restrict__ row,
+                                         int d) {
+    float acc = 0.f;
+    for (int e = 0; e < d; ++e) acc = fmaf(a_smem[e], to_f(row[e]), acc);
+    return acc;
+}
+
+struct RowCtx {
+    const int32_t *perm, *seg_lo, *seg_hi;
+    int n_valid, view;
+};
+
+__device__ __forceinline__ RowCtx row_ctx(const ViewPlan &rowv, const ViewPlan &colv,
+                                          const uint8_t *head_view, const int32_t *n_valid, int b,
+                                          int h, int N) {
+    RowCtx c;
+    c.view = head_view[h];
+    const ViewPlan &vp = c.view ? colv : rowv;
+    c.perm = vp.perm + (size_t)b * N;
+    c.seg_lo = vp.seg_lo + (size_t)b * N;
+    c.seg_hi = vp.seg_hi + (size_t)b * N;
+    c.n_valid = n_valid[b];
+    return c;
+}
+
+// ---------------------------------------------------------------------------------- forward
+template <typename T>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__restrict__ V,
+                T *__restrict__ O, float *__restrict__ LSE, ViewPlan rowv, ViewPlan colv,
+                const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
+                int P, int d, float scale) {
+    __shared__ float s_q[kWarpsPerBlock][kMaxD];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * kWarpsPerBlock + warp;
+    const int h = blockIdx.y, b = blockIdx.z, H = gridDim.y;
+    if (t >= N) return;
+    const RowCtx c = row_ctx(rowv, colv, head_view, n_valid, b, h, N);
+    const size_t bh = ((size_t)b * H + h) * N;
+    const int k = c.perm[t];
+    T *o_row = O + (bh + k) * d;
+    if (t >= c.n_valid) {  // padding query row
+        for (int e = lane; e < d; e += 32) from_f(o_row[e], 0.f);
+        if (lane == 0) LSE[bh + k] = -INFINITY;
+        return;
+    }
+    for (int e = lane; e < d; e += 32) s_q[warp][e] = to_f(Q[(bh + k) * d + e]);
+    __syncwarp();
+
+    float m = -INFINITY, l = 0.f, acc[kAccPerLane];
+#pragma unroll
+    for (int i = 0; i < kAccPerLane; ++i) acc[i] = 0.f;
+
+    const int lo = max(c.seg_lo[t], P), hi = c.seg_hi[t];
+    for (int range = 0; range < 2; ++range) {
+        const int j_begin = range ? lo : 0, j_end = range ? hi : P;
+        for (int j0 = j_begin; j0 < j_end; j0 += 32) {
+            const int j = j0 + lane;
+            const bool on = j < j_end;
+            const int kj = on ? c.perm[j] : 0;
+            float s = on ? scale * dot_row(s_q[warp], K + (bh + kj) * d, d) : -INFINITY;
+            const float m_new = fmaxf(m, warp_max(s));
+            const float p = on ? expf(s - m_new) : 0.f;
+            const float alpha = expf(m - m_new);  // m = -inf on the first step gives 0
+            l = l * alpha + warp_sum(p);
+            m = m_new;
+#pragma unroll
+            for (int i = 0; i < kAccPerLane; ++i) acc[i] *= alpha;
+            const int n_here = min(32, j_end - j0);
+            for (int jj = 0; jj < n_here; ++jj) {
+                const float pj = __shfl_sync(0xffffffffu, p, jj);
+                const int vj = __shfl_sync(0xffffffffu, kj, jj);
+                const T *v_row = V + (bh + vj) * d;
+#pragma unroll
+                for (int i = 0; i < kAccPerLane; ++i) {
+                    const int e = lane + 32 * i;
+                    if (e < d) acc[i] = fmaf(pj, to_f(v_row[e]), acc[i]);
+                }
+            }
+        }
+    }
+    const float inv_l = 1.f / l;  // every valid row attends at least to itself, so l > 0
+#pragma unroll
+    for (int i = 0; i < kAccPerLane; ++i) {
+        const int e = lane + 32 * i;
+        if (e < d) from_f(o_row[e], acc[i] * inv_l);
+    }
+    if (lane == 0) LSE[bh + k] = m + logf(l);
+}
+
+// ---------------------------------------------------------------------------------- backward
+// D_k = sum_e dO_ke O_ke, original token order, one warp per row.
+template <typename T>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_rowdot_kernel(const T *__restrict__ dO, const T *__restrict__ O, float *__restrict__ D,
+                   size_t rows, int d) {
+    const size_t r = (size_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    float acc = 0.f;
+    for (int e = lane; e < d; e += 32) acc = fmaf(to_f(dO[r * d + e]), to_f(O[r * d + e]), acc);
+    acc = warp_sum(acc);
+    if (lane == 0) D[r] = acc;
+}
+
+// kDKV = false: the warp owns query row t and produces dQ_t = scale * sum_j dS_tj K_j.
+// kDKV = true : the warp owns key row t and produces dV_t = sum_k P_kt dO_k and
+//               dK_t = scale * sum_k dS_kt Q_k, looping over the queries k that attend to it.
+template <typename T, bool kDKV>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+simt_bwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__restrict__ V,
+                const T *__restrict__ dO, const float *__restrict__ LSE,
+                const float *__restrict__ D, T *__restrict__ dQ, T *__restrict__ dK,
+                T *__restrict__ dV, ViewPlan rowv, ViewPlan colv,
+                const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
+                int P, int d, float scale) {
+    __shared__ float s_a[kWarpsPerBlock][kMaxD];  // own q (dQ) or own k (dK/dV)
+    __shared__ float s_b[kWarpsPerBlock][kMaxD];  // own dO (dQ) or own v (dK/dV)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * kWarpsPerBlock + warp;
+    const int h = blockIdx.y, b = blockIdx.z, H = gridDim.y;
+    if (t >= N) return;
+    const RowCtx c = row_ctx(rowv, colv, head_view, n_valid, b, h, N);
+    const size_t bh = ((size_t)b * H + h) * N;
+    const int own = c.perm[t];
+    T *out0 = (kDKV ? dK : dQ) + (bh + own) * d;
+    T *out1 = kDKV ? dV + (bh + own) * d : nullptr;
+    if (t >= c.n_valid) {
+        for (int e = lane; e < d; e += 32) {
+            from_f(out0[e], 0.f);
+            if (kDKV) from_f(out1[e], 0.f);
+        }
+        return;
+    }
+    const T *a_src = (kDKV ? K : Q) + (bh + own) * d;
+    const T *b_src = (kDKV ? V : dO) + (bh + own) * d;
+    for (int e = lane; e < d; e += 32) {
+        s_a[warp][e] = to_f(a_src[e]);
+        s_b[warp][e] = to_f(b_src[e]);
+    }
+    __syncwarp();
+    float own_lse = 0.f, own_D = 0.f;
+    if (!kDKV) {
+        own_lse = LSE[bh + own];
+        own_D = D[bh + own];
+    }
+    float acc0[kAccPerLane], acc1[kAccPerLane];
+#pragma unroll
+    for (int i = 0; i < kAccPerLane; ++i) acc0[i] = acc1[i] = 0.f;
+
+    const int lo = max(c.seg_lo[t], P), hi = c.seg_hi[t];
+    for (int range = 0; range < 2; ++range) {
+        const int j_begin = range ? lo : 0, j_end = range ? hi : P;
+        for (int j0 = j_begin; j0 < j_end; j0 += 32) {
+            const int j = j0 + lane;
+            const bool on = j < j_end;
+            const int oj = on ? c.perm[j] : 0;  // original index of the other row
+            float p = 0.f, ds = 0.f;
+            if (on) {
+                // dQ: other row is a key  -> s = q_own . k_other, dP = dO_own . v_other
+                // dKV: other row is a query -> s = q_other . k_own, dP = dO_other . v_own
+                const T *x = (kDKV ? Q : K) + (bh + oj) * d;
+                const T *y = (kDKV ? dO : V) + (bh + oj) * d;
+                const float s = scale * dot_row(s_a[warp], x, d);
+                const float dp = dot_row(s_b[warp], y, d);
+                const float lse = kDKV ? LSE[bh + oj] : own_lse;
+                const float Dk = kDKV ? D[bh + oj] : own_D;
+                p = expf(s - lse);
+                ds = p * (dp - Dk);
+            }
+            const int n_here = min(32, j_end - j0);
+            for (int jj = 0; jj < n_here; ++jj) {
+                const float pj = __shfl_sync(0xffffffffu, p, jj);
+                const float dsj = __shfl_sync(0xffffffffu, ds, jj) * scale;
+                const int rj = __shfl_sync(0xffffffffu, oj, jj);
+                const T *x = (kDKV ? Q : K) + (bh + rj) * d;   // dK += ds q ; dQ += ds k
+                const T *y = dO + (bh + rj) * d;               // dV += p dO
+#pragma unroll
+                for (int i = 0; i < kAccPerLane; ++i) {
+                    const int e = lane + 32 * i;
+                    if (e < d) {
+                        acc0[i] = fmaf(dsj, to_f(x[e]), acc0[i]);
+                        if (kDKV) acc1[i] = fmaf(pj, to_f(y[e]), acc1[i]);
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kAccPerLane; ++i) {
+        const int e = lane + 32 * i;
+        if (e < d) {
+            from_f(out0[e], acc0[i]);
+            if (kDKV) from_f(out1[e], acc1[i]);
+        }
+    }
+}
+
+template <typename T>
+int simt_fwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *V, int d, float scale,
+               void *O, float *LSE, cudaStream_t st) {
+    dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
+    simt_fwd_kernel<T><<<grid, kWarpsPerBlock * 32, 0, st>>>(
+        (const T *)Q, (const T *)K, (const T *)V, (T *)O, LSE, pl->view[0], pl->view[1],
+        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->P, d, scale);
+    return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
+}
+
+template <typename T>
+int simt_bwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *V, const void *O,
+               const float *LSE, const void *dO, int d, float scale, void *dQ, void *dK, void *dV,
+               void *ws, cudaStream_t st) {
+    float *D = (float *)ws;
+    const size_t rows = (size_t)pl->B * pl->H * pl->N;
+    simt_rowdot_kernel<T><<<(unsigned)((rows + kWarpsPerBlock - 1) / kWarpsPerBlock),
+                            kWarpsPerBlock * 32, 0, st>>>((const T *)dO, (const T *)O, D, rows, d);
+    dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
+    simt_bwd_kernel<T, false><<<grid, kWarpsPerBlock * 32, 0, st>>>(
+        (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->P, d, scale);
+    simt_bwd_kernel<T, true><<<grid, kWarpsPerBlock * 32, 0, st>>>(
+        (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->P, d, scale);
+    return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
+}
+
+}  // namespace
+
+int simt_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d, int dtype,
+             float scale, void *O, float *LSE, cudaStream_t stream) {
+    if (d > kMaxD) return MATE_ERR_UNSUPPORTED;
+    return dtype == MATE_F32 ? simt_fwd_t<float>(plan, Q, K, V, d, scale, O, LSE, stream)
+                             : simt_fwd_t<__nv_bfloat16>(plan, Q, K, V, d, scale, O, LSE, stream);
+}
+
+size_t simt_bwd_workspace(const mate_plan_t *plan) {
+    return sizeof(float) * (size_t)plan->B * plan->H * plan->N;
+}
+
+int simt_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, const void *O,
+             const float *LSE, const void *dO, int d, int dtype, float scale, void *dQ, void *dK,
+             void *dV, void *workspace, cudaStream_t stream) {
+    if (d > kMaxD) return MATE_ERR_UNSUPPORTED;
+    return dtype == MATE_F32
+               ? simt_bwd_t<float>(plan, Q, K, V, O, LSE, dO, d, scale, dQ, dK, dV, workspace, stream)
+               : simt_bwd_t<__nv_bfloat16>(plan, Q, K, V, O, LSE, dO, d, scale, dQ, dK, dV,
+                                           workspace, stream);
+}
+
+}  // namespace mate
