@@ -72,7 +72,7 @@ void build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_o
                 FwdUnit u{};
                 u.q0 = q0;
                 u.nq = std::min(kTile, P - q0);
-                u.kA0 = 0;
+                u.kA_end = nv;
                 u.kA_n = ceil_div(nv, kTile);
                 tiles.push_back(u);
             }
@@ -82,10 +82,11 @@ void build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_o
                 u.nq = std::min(kTile, nv - q0);
                 const int lo_first = so[seg_of(q0)];
                 const int hi_last = so[seg_of(q0 + u.nq - 1) + 1];
-                u.kA0 = 0;
+                u.kA_end = P;
                 u.kA_n = ceil_div(P, kTile);
-                u.kB0 = std::max(lo_first, u.kA_n * kTile);
-                u.kB_n = hi_last > u.kB0 ? ceil_div(hi_last - u.kB0, kTile) : 0;
+                u.kB0 = lo_first;
+                u.kB_end = hi_last;
+                u.kB_n = ceil_div(hi_last - lo_first, kTile);
                 tiles.push_back(u);
             }
             for (int q0 = nv; q0 < N; q0 += kTile) {

@@ -11,21 +11,24 @@ namespace mate {
 
 constexpr int kTile = 128;  // query rows and key columns per tile of the tensor-core kernels
 
-// One unit of forward work for the tensor-core kernel: 128 consecutive query rows (view order) of
-// one (example, head) and the key tiles they visit.  Key tiles are 128 wide.  Range A starts at
-// view position 0 (the prefix block, or every valid key for prefix query rows); range B starts at
-// kB0 (the segments the query rows belong to).  The per-row rule
-//     j < P  ||  seg_lo[row] <= j < seg_hi[row]
-// decides which keys inside a visited tile count.
+// One unit of forward work for the tensor-core kernel: up to 128 consecutive query rows (view
+// order) of one (example, head) and the key tiles they visit.  Key tiles are up to 128 wide.
+//   range A = keys [0, kA_end): the prefix block for table rows (kA_end = P), every valid key for
+//             prefix rows (kA_end = n_valid).  Inside it a key j counts iff j < kA_end.
+//   range B = keys [kB0, kB_end): the union of the segments the query rows belong to (table rows
+//             only, kB0 >= P).  Inside it key j counts for a row iff seg_lo[row] <= j < seg_hi[row].
 struct FwdUnit {
     int32_t b, h;
     int32_t q0, nq;        // first query row (view order) and number of rows (<= 128)
-    int32_t kA0, kA_n;     // first key of range A and its number of tiles
-    int32_t kB0, kB_n;     // first key of range B and its number of tiles
+    int32_t kA_end, kA_n;  // range A: end key and number of 128-key tiles
+    int32_t kB0, kB_end;   // range B: first and end key
+    int32_t kB_n;          // range B: number of tiles
     int32_t part, n_parts; // split-key bookkeeping: this unit is part `part` of `n_parts`
     int32_t slot;          // partial-result slot in the workspace when n_parts > 1, else -1
     int32_t cost;          // key tiles visited (sort key, largest first)
+    int32_t pad_[3];
 };
+static_assert(sizeof(FwdUnit) == 64, "FwdUnit is read as four 16-byte words");
 
 struct ViewPlan {
     int32_t *perm = nullptr;      // [B, N]   view position -> original position
