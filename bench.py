@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Benchmark of the multi-view attention hot path (plan pre-computed; forward + backward per step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl mate|reference] [--workload long]
+
+One step = one mate_attn_fwd + one mate_attn_bwd over one synthetic batch of the named workload.
+Prints ONE JSON line.  With N > 1 (torchrun) every rank runs its own replica of the workload
+(the path has no exchange step); the time is the max over ranks, the value the sum of the work.
+`--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from workloads import tables  # noqa: E402
+
+METRIC = "MATE attn fwd+bwd useful-pair TFLOP/s at N=8192 (4*d flop/pair fwd, 10*d bwd)"
+UNIT = "TFLOP/s"
+N_BUFFER_SETS = 4
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (same workload; None until a capture exists)
+NCU_TRAFFIC_BYTES = {"tc_fwd_kernel": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background (read-only queries)."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.samples = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self, t0, t1):
+        rows = [s for (t, s) in self.samples if t0 <= t <= t1] or [s for (_, s) in self.samples[-3:]]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except (ValueError, IndexError):
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_step(cfg, rows, cols, vals, hv, scale):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.fwd(vals["Q"], vals["K"], vals["V"], rows, cols, cfg.P, hv, scale)
+    t1 = time.perf_counter()
+    oracle.bwd(vals["Q"], vals["K"], vals["V"], vals["dO"], rows, cols, cfg.P, hv, scale)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def pair_flops(cfg, pairs):
+    return 4.0 * cfg.d * pairs, 10.0 * cfg.d * pairs
+
+
+def run_reference(args, cfg):
+    """CPU oracle arm.  Each step is one forward + backward of a bounded sample of the workload:
+    the same table, a subset of the heads (always at least one row head and one column head),
+    chosen so that warmup + steps stay within a few minutes on the host cores."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows, cols, info = tables.make_structure(cfg, 1234)
+    vals = tables.make_values(cfg, info["N"], 5678)
+    hv = tables.head_view(cfg)
+    scale = 1.0 / np.sqrt(cfg.d)
+    row_heads = [h for h in range(cfg.H) if hv[h] == 0]
+    col_heads = [h for h in range(cfg.H) if hv[h] == 1]
+
+    def subset(k):  # k heads of each view (all heads of a view when it has fewer)
+        return sorted(row_heads[:k] + col_heads[:k])
+
+    def sample_of(hsel):
+        return {n: np.ascontiguousarray(v[:, hsel]) for n, v in vals.items()}, hv[hsel]
+
+    # calibrate on the smallest sample, then take the largest sample that fits the time budget
+    hsel = subset(1)
+    sv, shv = sample_of(hsel)
+    t0 = time.perf_counter()
+    oracle_step(cfg, rows, cols, sv, shv, scale)
+    t_small = time.perf_counter() - t0
+    budget = 150.0 / max(args.steps + args.warmup, 1)
+    k = max(1, min(max(len(row_heads), len(col_heads)), int(budget / max(t_small, 1e-9))))
+    if k > 1:
+        hsel = subset(k)
+        sv, shv = sample_of(hsel)
+    pairs = float(oracle.useful_pairs(rows, cols, cfg.P, shv).sum())
+    f_fwd, f_bwd = pair_flops(cfg, pairs)
+    for _ in range(args.warmup):
+        oracle_step(cfg, rows, cols, sv, shv, scale)
+    tf = tb = 0.0
+    for _ in range(args.steps):
+        a, b = oracle_step(cfg, rows, cols, sv, shv, scale)
+        tf += a
+        tb += b
+    t_step = (tf + tb) / args.steps
+    value = (f_fwd + f_bwd) / t_step / 1e12
+    sample = "%s workload (B=%d N=%d), heads %s of %d, fwd+bwd per step, fp64" % (
+        cfg.name, cfg.B, info["N"], hsel, cfg.H)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "H": cfg.H, "N": info["N"], "d": cfg.d, "P": cfg.P},
+        "fwd": {"ms": tf / args.steps * 1e3, "tflops": f_fwd / (tf / args.steps) / 1e12},
+        "bwd": {"ms": tb / args.steps * 1e3, "tflops": f_bwd / (tb / args.steps) / 1e12},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_mate(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2109_04312_b200 as mate
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    peaks = load_peaks()
+
+    # every rank builds its own replica of the workload (different seed per rank): no exchange step
+    rows, cols, info = tables.make_structure(cfg, 1234 + rank)
+    hv = tables.head_view(cfg)
+    N = info["N"]
+    scale = 1.0 / np.sqrt(cfg.d)
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    plan = mate.mate_plan(torch.from_numpy(rows).to(dev), torch.from_numpy(cols).to(dev), cfg.P, hv,
+                          cfg.n_rows, cfg.n_cols)
+    pairs = float(plan.useful_pairs().sum())
+    n_valid_tokens = float(sum(info["n_valid"]))
+    f_fwd, f_bwd = pair_flops(cfg, pairs)
+
+    host = tables.make_values(cfg, N, 5678 + rank)
+    pinned = {k: torch.from_numpy(v).to(tdt).pin_memory() for k, v in host.items()}
+    sets = []
+    for s in range(N_BUFFER_SETS):
+        d = {k: pinned[k].to(dev, non_blocking=True).clone() for k in ("Q", "K", "V", "dO")}
+        if s:
+            for k in d:  # distinct contents per set, same distribution
+                d[k] = d[k].roll(s, dims=2).contiguous()
+        d["O"] = torch.empty_like(d["Q"])
+        d["LSE"] = torch.empty((cfg.B, cfg.H, N), dtype=torch.float32, device=dev)
+        sets.append(d)
+    torch.cuda.synchronize()
+    set_bytes = sum(t.numel() * t.element_size() for t in sets[0].values()) + 3 * sets[0]["Q"].numel() * 2
+
+    def step(d):
+        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, out=d["O"], lse=d["LSE"])
+        return mate.mate_attn_bwd(plan, d["Q"], d["K"], d["V"], d["O"], d["LSE"], d["dO"], scale)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+
+    for i in range(args.warmup):
+        step(sets[i % N_BUFFER_SETS])
+    torch.cuda.synchronize()
+    plan.status()
+
+    # ---- device-resident timing: K steps, CUDA events on the launching (current) stream
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    for i in range(K):
+        d = sets[i % N_BUFFER_SETS]
+        ev[i][0].record()
+        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, out=d["O"], lse=d["LSE"])
+        ev[i][1].record()
+        mate.mate_attn_bwd(plan, d["Q"], d["K"], d["V"], d["O"], d["LSE"], d["dO"], scale)
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t_wall1 = time.time()
+    plan.status()
+    total_ms = ev[0][0].elapsed_time(ev[K - 1][2])
+    fwd_ms = np.asarray([e[0].elapsed_time(e[1]) for e in ev])
+    bwd_ms = np.asarray([e[1].elapsed_time(e[2]) for e in ev])
+
+    # ---- end-to-end timing: pinned host inputs -> device, forward + backward, results -> host
+    e2e_steps = max(3, min(K, 20))
+    res_host = {k: torch.empty_like(pinned["Q"]) for k in ("O", "dQ", "dK", "dV")}
+    lse_host = torch.empty((cfg.B, cfg.H, N), dtype=torch.float32).pin_memory()
+    for k in res_host:
+        res_host[k] = res_host[k].pin_memory()
+    h2d = sum(pinned[k].numel() * pinned[k].element_size() for k in ("Q", "K", "V", "dO"))
+    d2h = sum(t.numel() * t.element_size() for t in res_host.values()) + lse_host.numel() * 4
+
+    def e2e_step(d):
+        for k in ("Q", "K", "V", "dO"):
+            d[k].copy_(pinned[k], non_blocking=True)
+        dQ, dK, dV = step(d)
+        res_host["O"].copy_(d["O"], non_blocking=True)
+        lse_host.copy_(d["LSE"], non_blocking=True)
+        res_host["dQ"].copy_(dQ, non_blocking=True)
+        res_host["dK"].copy_(dK, non_blocking=True)
+        res_host["dV"].copy_(dV, non_blocking=True)
+
+    e2e_step(sets[0])
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(sets[i % N_BUFFER_SETS])
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    if rank == 0:
+        sampler.stop()
+
+    times = torch.tensor([total_ms, float(np.median(fwd_ms)), float(np.median(bwd_ms)), e2e_ms,
+                          float(fwd_ms.min()), float(bwd_ms.min())], dtype=torch.float64, device=dev)
+    work = torch.tensor([pairs, n_valid_tokens], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+        dist.all_reduce(work, op=dist.ReduceOp.SUM)
+    total_ms, fwd_med, bwd_med, e2e_ms, fwd_min, bwd_min = times.tolist()
+    pairs_all, tokens_all = work.tolist()
+    ff, fb = pair_flops(cfg, pairs_all)
+    ms_per_step = total_ms / K
+
+    if rank == 0:
+        value = (ff + fb) / (ms_per_step * 1e-3) / 1e12
+        fwd_tflops = ff / (fwd_med * 1e-3) / 1e12
+        bwd_tflops = fb / (bwd_med * 1e-3) / 1e12
+        # roofline of the forward tensor-core kernel (one launch = the whole forward of one rank)
+        fwd_tflops_rank = f_fwd / (float(np.mean(fwd_ms)) * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "H": cfg.H, "N": N, "d": cfg.d, "P": cfg.P,
+                       "useful_pairs": pairs_all, "dense_pairs": float(world * cfg.B * cfg.H * N * N),
+                       "l2": "rotating %d buffer sets of %.0f MB (> 126 MB L2)" % (N_BUFFER_SETS, set_bytes / 1e6),
+                       "plan": "pre-computed, outside the timed region"},
+            "fwd": {"ms_median": fwd_med, "ms_min": fwd_min, "tflops": fwd_tflops,
+                    "frac_of_bf16_peak": fwd_tflops / (peaks["bf16_tflops"] * world),
+                    "tokens_per_s": tokens_all / (fwd_med * 1e-3)},
+            "bwd": {"ms_median": bwd_med, "ms_min": bwd_min, "tflops": bwd_tflops,
+                    "frac_of_bf16_peak": bwd_tflops / (peaks["bf16_tflops"] * world),
+                    "tokens_per_s": tokens_all / (bwd_med * 1e-3)},
+            "tokens_per_s": tokens_all / (ms_per_step * 1e-3),
+            "roofline": {"kernel": "tc_fwd_kernel", "bound": "tensor", "achieved": fwd_tflops_rank,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": fwd_tflops_rank / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                         "traffic": NCU_TRAFFIC_BYTES["tc_fwd_kernel"]},
+            "e2e": {"value": (ff + fb) / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": K * 4,
+            "clocks": sampler.summary(t_wall0, t_wall1),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            sub = cfg
+            tf, tb = oracle_step(sub, rows, cols, host, hv, scale)
+            import oracle
+            line["cpu_baseline"] = {
+                "value": (f_fwd + f_bwd) / (tf + tb) / 1e12, "unit": UNIT, "cores": oracle.num_threads(),
+                "kind": "oracle", "fwd_s": tf, "bwd_s": tb,
+                "sample": "whole %s workload once (B=%d H=%d N=%d), fwd+bwd, fp64" % (cfg.name, cfg.B, cfg.H, N)}
+        print(json.dumps(line), flush=True)
+    plan.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="mate", choices=["mate", "reference"])
+    ap.add_argument("--workload", default="long", choices=sorted(tables.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = tables.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_mate(args, cfg)
+
+
+if __name__ == "__main__":
+    main()
