@@ -47,7 +47,8 @@ enum {
     MATE_ERR_CUDA = -4,        /* a CUDA runtime call failed (the CUDA error is left in place)      */
     MATE_ERR_TIMEOUT = -5,     /* a bounded wait inside a kernel expired (see mate_plan_status)     */
     MATE_ERR_NOMEM = -6,       /* host or device allocation failed                                  */
-    MATE_ERR_WORKSPACE = -7    /* workspace pointer null or smaller than mate_attn_workspace_bytes  */
+    MATE_ERR_WORKSPACE = -7,   /* workspace pointer null or smaller than mate_attn_workspace_bytes  */
+    MATE_ERR_TOO_LARGE = -8    /* problem exceeds the built-in scratch of mate_attn_bwd_noalloc      */
 };
 
 enum { MATE_BF16 = 0, MATE_F32 = 1 };          /* element type of Q, K, V, O, dO, dQ, dK, dV */
@@ -123,6 +124,31 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
                   const void *O, const float *LSE, const void *dO, int d, int dtype, float scale,
                   void *dQ, void *dK, void *dV, void *workspace, size_t workspace_bytes,
                   unsigned flags, void *stream);
+
+/* Backward for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a serving or training loop whose
+ * framework has handed all device memory to its own pool, a latency-critical section where the
+ * device-wide synchronisation of cudaMalloc/cudaFree is not acceptable, or a plug-in that gets
+ * tensors but no allocator.  Such a caller cannot create the workspace mate_attn_bwd asks for.
+ *
+ * Same arguments, results and rules as mate_attn_bwd with flags = MATE_IMPL_SIMT, minus the
+ * workspace: the scratch (one float per (example, head, position)) lives in a 4 MiB array that is
+ * part of the library itself, so every GPU that loads libmate holds it until the process exits.
+ * The call makes no cudaMalloc, cudaFree or other allocating call.
+ *
+ *   limit       B * H * N <= 1,048,576; larger problems return MATE_ERR_TOO_LARGE and launch nothing
+ *   first call  the first call on each device looks up the array's device address (with that
+ *               device current); make that first call outside any stream capture
+ *   sharing     all calls on a device use the same array.  Its contents are left over from the
+ *               previous call; the kernels overwrite every element they later read, so nothing
+ *               depends on them.  Two calls that overlap on the GPU (different streams) race on
+ *               the array: serialise them.
+ * The plan is an input like the tensors; create it ahead of time with mate_plan. */
+int mate_attn_bwd_noalloc(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
+                          const void *O, const float *LSE, const void *dO, int d, int dtype,
+                          float scale, void *dQ, void *dK, void *dV, void *stream);
 
 #ifdef __cplusplus
 }

@@ -54,6 +54,8 @@ def _load():
     lib.mate_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, sz, u32, vp]
     lib.mate_attn_bwd.restype = i32
     lib.mate_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, vp, sz, u32, vp]
+    lib.mate_attn_bwd_noalloc.restype = i32
+    lib.mate_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -206,4 +208,26 @@ def mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale=None, impl=IMPL_AUTO, workspa
                                      C.c_void_p(ws.data_ptr()) if ws is not None else None,
                                      ws.numel() if ws is not None else 0, impl, _stream()),
                "mate_attn_bwd")
+    return dQ, dK, dV
+
+
+def mate_attn_bwd_noalloc(plan, Q, K, V, O, LSE, dO, dQ, dK, dV, scale=None):
+    """Backward for callers that may not allocate device memory (for example inside a loop whose
+    framework owns every byte of the device): the caller passes the three output tensors and the
+    library uses its built-in scratch array, so neither this function nor the C entry point
+    allocates anything.  B*H*N is limited to 1,048,576.  Calls must not overlap on the GPU."""
+    B, H, N, d = Q.shape
+    if (B, H, N) != (plan.B, plan.H, plan.N):
+        raise ValueError("tensor shapes do not match the plan")
+    for t in (K, V, O, dO, dQ, dK, dV):
+        if t.shape != Q.shape or t.dtype != Q.dtype:
+            raise ValueError("K, V, O, dO, dQ, dK, dV must match Q in shape and dtype")
+    if scale is None:
+        scale = 1.0 / float(d) ** 0.5
+    with torch.cuda.device(Q.device):
+        _check(_load().mate_attn_bwd_noalloc(plan._h, _dev(Q, "Q"), _dev(K, "K"), _dev(V, "V"),
+                                             _dev(O, "O"), _dev(LSE, "LSE"), _dev(dO, "dO"), d,
+                                             _dtype_code(Q), float(scale), _dev(dQ, "dQ"),
+                                             _dev(dK, "dK"), _dev(dV, "dV"), _stream()),
+               "mate_attn_bwd_noalloc")
     return dQ, dK, dV

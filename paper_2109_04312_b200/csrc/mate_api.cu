@@ -136,6 +136,7 @@ const char *mate_status_string(int status) {
         case MATE_ERR_TIMEOUT: return "bounded device wait expired";
         case MATE_ERR_NOMEM: return "out of memory";
         case MATE_ERR_WORKSPACE: return "workspace missing or too small";
+        case MATE_ERR_TOO_LARGE: return "B*H*N exceeds the built-in scratch of mate_attn_bwd_noalloc";
         default: return "unknown status";
     }
 }

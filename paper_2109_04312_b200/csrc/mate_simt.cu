@@ -9,11 +9,19 @@
 // attend to key t are the same two ranges; dK/dV therefore need no atomics.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "mate_internal.h"
 
 namespace mate {
 
 namespace {
+
+// Built-in scratch of mate_attn_bwd_noalloc: one float per (example, head, position) for the row
+// dots D.  It is part of the library image, so every GPU that loads the library holds these
+// 4 MiB until the process exits.
+constexpr size_t kNoAllocMaxRows = size_t(1) << 20;
+static __device__ __align__(256) float g_noalloc_rowdot[kNoAllocMaxRows];
 
 constexpr int kWarpsPerBlock = 4;
 constexpr int kMaxD = 128;
@@ -286,3 +294,43 @@ int simt_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *
 }
 
 }  // namespace mate
+
+// Allocation-free backward (see mate.h).  The name g_noalloc_rowdot is only a host-side handle
+// here; the address the kernels need comes from cudaGetSymbolAddress, looked up once per device
+// with that device current.
+extern "C" int mate_attn_bwd_noalloc(const mate_plan_t *plan, const void *Q, const void *K,
+                                     const void *V, const void *O, const float *LSE,
+                                     const void *dO, int d, int dtype, float scale, void *dQ,
+                                     void *dK, void *dV, void *stream) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static float *scratch_of_device[kMaxDevices] = {};
+
+    if (!plan || !Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return MATE_ERR_INVALID_ARG;
+    if (dtype != MATE_BF16 && dtype != MATE_F32) return MATE_ERR_UNSUPPORTED;
+    if (d <= 0 || d % 8 != 0 || d > mate::kMaxD) return MATE_ERR_UNSUPPORTED;
+    const void *ptrs[] = {Q, K, V, O, LSE, dO, dQ, dK, dV};
+    for (const void *p : ptrs)
+        if (reinterpret_cast<uintptr_t>(p) & 15u) return MATE_ERR_ALIGNMENT;
+    const size_t rows = (size_t)plan->B * plan->H * plan->N;
+    if (rows > mate::kNoAllocMaxRows) return MATE_ERR_TOO_LARGE;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MATE_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return MATE_ERR_UNSUPPORTED;
+    float *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!scratch_of_device[dev]) {
+            float *p = nullptr;
+            if (cudaGetSymbolAddress((void **)&p, mate::g_noalloc_rowdot) != cudaSuccess || !p)
+                return MATE_ERR_CUDA;
+            scratch_of_device[dev] = p;
+        }
+        scratch = scratch_of_device[dev];
+    }
+    // every element of D that the backward kernels read is written by the row-dot kernel of the
+    // same call first, so nothing in the shared array has to start at zero
+    return mate::simt_bwd(plan, Q, K, V, O, LSE, dO, d, dtype, scale, dQ, dK, dV, scratch,
+                          (cudaStream_t)stream);
+}
