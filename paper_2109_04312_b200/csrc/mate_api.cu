@@ -30,7 +30,7 @@ struct Carver {
     }
 };
 
-void carve(mate_plan_t *pl, char *base, size_t *total, int max_units) {
+void carve(mate_plan_t *pl, char *base, size_t *total) {
     Carver c(base);
     const size_t BN = (size_t)pl->B * pl->N;
     for (int v = 0; v < 2; ++v) {
@@ -46,80 +46,185 @@ void carve(mate_plan_t *pl, char *base, size_t *total, int max_units) {
     pl->n_valid_dev = c.take<int32_t>(pl->B);
     pl->status_dev = c.take<int32_t>(4);
     pl->head_view_dev = c.take<uint8_t>(pl->H);
-    pl->fwd_units_dev = c.take<FwdUnit>(max_units);
-    pl->bwd_units_dev = c.take<FwdUnit>(max_units);
     *total = align_up(c.off, 256);
 }
 
-// Tile work-list of the tensor-core kernels, built on the host from the segment offsets.
-// `symmetric` units are reused by the backward kernels (the pattern is symmetric, so the key tiles
-// a query tile visits are also the query tiles a key tile is visited by).
-void build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_off_host) {
-    std::vector<FwdUnit> units;
+// Work-list of the tensor-core forward, built on the host from the segment offsets, then spread
+// over the CTAs of a persistent kernel so that every CTA gets about the same amount of softmax
+// work (longest-processing-time-first: units by decreasing cost, each to the least loaded CTA).
+//
+// Cost model: the exponentials are the inner limit of the kernel, and a warp (32 query rows)
+// evaluates them 32 key columns at a time, so the cost of a unit is the number of (warp, 32-column
+// chunk) pairs it visits plus a constant per half for loading Q and storing O.
+constexpr int kChunk = 32;
+constexpr int kCostPerHalf = 12;
+
+struct UnitCost {
+    FwdUnit u;
+    int64_t cost;
+};
+
+int64_t half_cost(const FwdUnit &u, int h, const int32_t *so, int S) {
+    const int rows = std::min(kTile, u.nq - h * kTile);
+    if (rows <= 0) return 0;
+    int64_t c = kCostPerHalf;
+    const int n_warps = ceil_div(rows, 32);
+    c += (int64_t)n_warps * ceil_div(std::max(u.kA_end - u.kA0, 0), kChunk);
+    if (u.kB_end > u.kB0) {
+        auto seg_of = [&](int t) { return (int)(std::upper_bound(so, so + S, t) - so) - 1; };
+        for (int w = 0; w < n_warps; ++w) {
+            const int t0 = u.q0 + h * kTile + w * 32;
+            const int t1 = std::min(t0 + 32, u.q0 + h * kTile + rows) - 1;
+            const int lo = so[seg_of(t0)], hi = so[seg_of(t1) + 1];
+            c += ceil_div(hi - lo, kChunk) + 1;  // + 1: chunks are aligned to the tile, not to lo
+        }
+    }
+    return c;
+}
+
+int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_off_host) {
     const int P = pl->P, N = pl->N;
-    for (int v = 0; v < 2; ++v) {
-        const ViewPlan &vp = pl->view[v];
-        if (vp.n_heads == 0) continue;
-        const int S = vp.max_id + 2;
-        for (int b = 0; b < pl->B; ++b) {
-            const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
-            const int nv = pl->n_valid[b];
-            std::vector<FwdUnit> tiles;
-            auto seg_of = [&](int t) {  // segment index s with so[s] <= t < so[s+1]
-                return (int)(std::upper_bound(so, so + S, t) - so) - 1;
-            };
-            for (int q0 = 0; q0 < P; q0 += kTile) {
-                FwdUnit u{};
-                u.q0 = q0;
-                u.nq = std::min(kTile, P - q0);
-                u.kA_end = nv;
-                u.kA_n = ceil_div(nv, kTile);
-                tiles.push_back(u);
-            }
-            for (int q0 = P; q0 < nv; q0 += kTile) {
-                FwdUnit u{};
-                u.q0 = q0;
-                u.nq = std::min(kTile, nv - q0);
-                const int lo_first = so[seg_of(q0)];
-                const int hi_last = so[seg_of(q0 + u.nq - 1) + 1];
-                u.kA_end = P;
-                u.kA_n = ceil_div(P, kTile);
-                u.kB0 = lo_first;
-                u.kB_end = hi_last;
-                u.kB_n = ceil_div(hi_last - lo_first, kTile);
-                tiles.push_back(u);
-            }
-            for (int q0 = nv; q0 < N; q0 += kTile) {
-                FwdUnit u{};
-                u.q0 = q0;
-                u.nq = std::min(kTile, N - q0);
-                tiles.push_back(u);
-            }
-            for (int h = 0; h < pl->H; ++h) {
-                if (pl->head_view[h] != v) continue;
-                for (FwdUnit u : tiles) {
-                    u.b = b;
-                    u.h = h;
-                    u.part = 0;
+    std::vector<UnitCost> all;
+    // pass 1: units without splitting, to learn the total cost; pass 2 splits the long prefix units
+    int64_t split_tiles = 1 << 30;
+    for (int pass = 0; pass < 2; ++pass) {
+        all.clear();
+        pl->n_fwd_slots = 0;
+        pl->fwd_ws_bytes = 0;
+        int64_t total = 0;
+        for (int v = 0; v < 2; ++v) {
+            const ViewPlan &vp = pl->view[v];
+            if (vp.n_heads == 0) continue;
+            const int S = vp.max_id + 2;
+            for (int b = 0; b < pl->B; ++b) {
+                const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
+                const int nv = pl->n_valid[b];
+                auto seg_of = [&](int t) { return (int)(std::upper_bound(so, so + S, t) - so) - 1; };
+                std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
+                for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
+                    FwdUnit u{};
+                    u.q0 = q0;
+                    u.nq = std::min(mate::kUnitRows, P - q0);
+                    const int n_tiles = ceil_div(nv, kTile);
+                    const int want = ceil_div(n_tiles, (int)std::min<int64_t>(split_tiles, n_tiles));
+                    const int per = ceil_div(n_tiles, want);
+                    const int n_parts = ceil_div(n_tiles, per);  // every part holds at least one tile
+                    for (int part = 0; part < n_parts; ++part) {
+                        FwdUnit w = u;
+                        w.kA0 = part * per * kTile;
+                        w.kA_end = std::min(nv, (part + 1) * per * kTile);
+                        if (w.kA_end <= w.kA0) continue;
+                        w.n_parts = n_parts;
+                        w.part = part;
+                        proto.push_back({w, 0});
+                    }
+                }
+                for (int q0 = P; q0 < nv; q0 += mate::kUnitRows) {  // table rows: prefix + own segments
+                    FwdUnit u{};
+                    u.q0 = q0;
+                    u.nq = std::min(mate::kUnitRows, nv - q0);
+                    u.kA0 = 0;
+                    u.kA_end = P;
+                    u.kB0 = so[seg_of(q0)];
+                    u.kB_end = so[seg_of(q0 + u.nq - 1) + 1];
+                    for (int h = 0; h < 2; ++h) {
+                        const int r0 = q0 + h * kTile, r1 = std::min(q0 + u.nq, r0 + kTile) - 1;
+                        if (r1 < r0) continue;
+                        u.lo[h] = so[seg_of(r0)];
+                        u.hi[h] = so[seg_of(r1) + 1];
+                    }
                     u.n_parts = 1;
-                    u.slot = -1;
-                    u.cost = u.kA_n + u.kB_n;
-                    units.push_back(u);
+                    proto.push_back({u, 0});
+                }
+                for (int q0 = nv; q0 < N; q0 += mate::kUnitRows) {  // padding rows: no key at all
+                    FwdUnit u{};
+                    u.q0 = q0;
+                    u.nq = std::min(mate::kUnitRows, N - q0);
+                    u.n_parts = 1;
+                    proto.push_back({u, 0});
+                }
+                for (auto &pc : proto) pc.cost = half_cost(pc.u, 0, so, S) + half_cost(pc.u, 1, so, S);
+                for (int h = 0; h < pl->H; ++h) {
+                    if (pl->head_view[h] != v) continue;
+                    int slot = -1;
+                    for (UnitCost pc : proto) {
+                        pc.u.b = b;
+                        pc.u.h = h;
+                        pc.u.ctr = -1;
+                        if (pc.u.n_parts > 1) {
+                            if (pc.u.part == 0) {
+                                slot = pl->n_fwd_slots++;
+                            }
+                            pc.u.ctr = slot;
+                            pc.u.ws_off = (int32_t)((pl->fwd_ws_bytes + pc.u.part * mate::kPartialBytes) >> 10);
+                            if (pc.u.part == pc.u.n_parts - 1) pl->fwd_ws_bytes += pc.u.n_parts * mate::kPartialBytes;
+                        }
+                        total += pc.cost;
+                        all.push_back(pc);
+                    }
                 }
             }
         }
+        if (pass == 0) {
+            // a split part should cost about a quarter of a CTA's share (never below two key tiles)
+            const int64_t share = total / std::max(pl->n_ctas, 1);
+            const int64_t part_cost = std::max<int64_t>(share / 4, 1);
+            // cost of one key tile of a full prefix unit: 8 warps x 4 chunks
+            split_tiles = std::max<int64_t>(2, part_cost / 32);
+        }
     }
-    std::stable_sort(units.begin(), units.end(),
-                     [](const FwdUnit &a, const FwdUnit &b) { return a.cost > b.cost; });
-    pl->fwd_units = std::move(units);
-    pl->n_fwd_units = (int)pl->fwd_units.size();
-    pl->n_fwd_slots = 0;
-}
+    static_assert(mate::kPartialBytes % 1024 == 0, "ws_off counts KiB");
 
-int max_units_bound(int B, int N, int P, int H) {
-    // per (b, h): prefix tiles + table tiles + padding tiles, each at most ceil(.../128) + 1
-    const int per = ceil_div(P, kTile) + 2 * (ceil_div(N, kTile) + 1);
-    return B * H * per;
+    // longest first, each to the least loaded CTA
+    std::stable_sort(all.begin(), all.end(), [](const UnitCost &a, const UnitCost &b) { return a.cost > b.cost; });
+    const int n_ctas = std::max(pl->n_ctas, 1);
+    std::vector<std::vector<int>> mine(n_ctas);
+    std::vector<std::pair<int64_t, int>> heap;  // (load, cta) min-heap
+    for (int c = 0; c < n_ctas; ++c) heap.push_back({0, c});
+    auto cmp = [](const std::pair<int64_t, int> &a, const std::pair<int64_t, int> &b) { return a > b; };
+    std::make_heap(heap.begin(), heap.end(), cmp);
+    for (int i = 0; i < (int)all.size(); ++i) {
+        std::pop_heap(heap.begin(), heap.end(), cmp);
+        auto &top = heap.back();
+        mine[top.second].push_back(i);
+        top.first += all[i].cost;
+        std::push_heap(heap.begin(), heap.end(), cmp);
+    }
+    pl->fwd_units.clear();
+    pl->fwd_cta_begin.assign(n_ctas + 1, 0);
+    for (int c = 0; c < n_ctas; ++c) {
+        pl->fwd_cta_begin[c] = (int32_t)pl->fwd_units.size();
+        for (int i : mine[c]) pl->fwd_units.push_back(all[i].u);
+    }
+    pl->fwd_cta_begin[n_ctas] = (int32_t)pl->fwd_units.size();
+    pl->n_fwd_units = (int)pl->fwd_units.size();
+    if (getenv("MATE_LOG")) {
+        int64_t mx = 0, sum = 0;
+        for (auto &hc : heap) {
+            mx = std::max(mx, hc.first);
+            sum += hc.first;
+        }
+        fprintf(stderr, "[mate] forward work-list: %d units, %d split slots, %d CTAs, cost max %lld mean %.1f, "
+                        "split at %lld key tiles, workspace %zu bytes\n",
+                pl->n_fwd_units, pl->n_fwd_slots, n_ctas, (long long)mx, (double)sum / n_ctas,
+                (long long)split_tiles, pl->fwd_ws_bytes);
+    }
+
+    // device copy: units, CTA offsets, arrival counters (zeroed once; the kernel resets them)
+    Carver c(nullptr);
+    c.take<FwdUnit>(pl->n_fwd_units);
+    c.take<int32_t>(n_ctas + 1);
+    c.take<int32_t>(8 * (size_t)std::max(pl->n_fwd_slots, 1));
+    const size_t bytes = align_up(c.off, 256);
+    if (cudaMalloc(&pl->work_block, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return MATE_ERR_NOMEM;
+    }
+    Carver d((char *)pl->work_block);
+    pl->fwd_units_dev = d.take<FwdUnit>(pl->n_fwd_units);
+    pl->fwd_cta_begin_dev = d.take<int32_t>(n_ctas + 1);
+    pl->fwd_counters_dev = d.take<int32_t>(8 * (size_t)std::max(pl->n_fwd_slots, 1));
+    return MATE_OK;
 }
 
 }  // namespace
@@ -144,6 +249,7 @@ const char *mate_status_string(int status) {
 int mate_plan_destroy(mate_plan_t *plan) {
     if (!plan) return MATE_OK;
     if (plan->dev_block) cudaFree(plan->dev_block);
+    if (plan->work_block) cudaFree(plan->work_block);
     delete plan;
     return MATE_OK;
 }
@@ -172,15 +278,22 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
     pl->view[1].max_id = max_col_id;
     for (int h = 0; h < H; ++h) pl->view[head_view[h]].n_heads++;
 
-    const int max_units = max_units_bound(B, N, prefix_len, H);
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&pl->n_ctas, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            delete pl;
+            return MATE_ERR_CUDA;
+        }
+    }
     size_t total = 0;
-    carve(pl, nullptr, &total, max_units);
+    carve(pl, nullptr, &total);
     if (cudaMalloc(&pl->dev_block, total) != cudaSuccess) {
         cudaGetLastError();
         delete pl;
         return MATE_ERR_NOMEM;
     }
-    carve(pl, (char *)pl->dev_block, &total, max_units);
+    carve(pl, (char *)pl->dev_block, &total);
 
     int rc = MATE_OK;
     int32_t status_host[4] = {0, 0, 0, 0};
@@ -224,15 +337,21 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
         }
     }
 
-    build_units(pl, seg_off_host);
-    if (pl->n_fwd_units > max_units) {  // cannot happen; guards the device array
+    rc = build_units(pl, seg_off_host);
+    if (rc != MATE_OK) {
         mate_plan_destroy(pl);
-        return MATE_ERR_INVALID_ARG;
+        return rc;
     }
-    if (pl->n_fwd_units > 0 &&
-        (cudaMemcpyAsync(pl->fwd_units_dev, pl->fwd_units.data(),
-                         sizeof(FwdUnit) * pl->n_fwd_units, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-         cudaStreamSynchronize(st) != cudaSuccess)) {
+    bool up = cudaMemsetAsync(pl->fwd_counters_dev, 0, sizeof(int32_t) * 8 * (size_t)std::max(pl->n_fwd_slots, 1),
+                              st) == cudaSuccess;
+    up = up && cudaMemcpyAsync(pl->fwd_cta_begin_dev, pl->fwd_cta_begin.data(),
+                               sizeof(int32_t) * pl->fwd_cta_begin.size(), cudaMemcpyHostToDevice,
+                               st) == cudaSuccess;
+    if (pl->n_fwd_units > 0)
+        up = up && cudaMemcpyAsync(pl->fwd_units_dev, pl->fwd_units.data(), sizeof(FwdUnit) * pl->n_fwd_units,
+                                   cudaMemcpyHostToDevice, st) == cudaSuccess;
+    up = up && cudaStreamSynchronize(st) == cudaSuccess;
+    if (!up) {
         mate_plan_destroy(pl);
         return MATE_ERR_CUDA;
     }

@@ -1,18 +1,23 @@
 // Tensor-core forward of multi-view attention (head formula and pattern of Section 3) for bf16,
-// d = 64, on sm_100a: tcgen05 MMAs with accumulators in TMEM, operands gathered into 128-byte
-// swizzled shared memory in the head's view order (Section 3.1: per-head traversal order).
+// d = 64, on sm_100a.  One persistent, warp-specialised CTA per SM walks the units that
+// mate_plan assigned to it (see FwdUnit): 256 query rows of one (example, head) in the head's view
+// order (Section 3.1: per-head traversal order) against the key tiles those rows may attend.
 //
-// One CTA (128 threads, thread r = query row r of the tile) walks a list of units (see FwdUnit).
-// For every key tile of a unit:
-//     S = Q K^T            tcgen05.mma, M = 128, N = tile width rounded to 16, K = 64  -> TMEM
-//     online softmax       one thread per row reads its S row from TMEM (two passes: max, then
-//                          exp2 / row sum), writes P as bf16 into swizzled shared memory
-//     O += P V             tcgen05.mma, M = 128, N = 64, K = tile width; O stays in TMEM and is
-//                          rescaled only when a row's running max grows by more than 2^8
-// Gather is fused into the loads (each 128-byte row is fetched by its view-order index with
-// cp.async), scatter into the epilogue (each thread stores its row at the original position).
-// Two CTAs share an SM (256 of 512 TMEM columns and ~98 KB of shared memory each), so one CTA's
-// softmax overlaps the other's MMAs.
+//   warps 0-3   softmax of half 0 (query rows 0..127 of the unit), one thread per row
+//   warps 4-7   softmax of half 1 (rows 128..255)
+//   warp  8     one thread issues every tcgen05.mma
+//   warps 9-11  loaders: gather Q, K, V rows by view-order index into 128-byte swizzled shared
+//               memory with 16-byte cp.async (the gather of Section 3.1 fused into the loads)
+//
+// Per key tile and half:   S = Q K^T  (tcgen05.mma, M = 128, N <= 128, K = 64, accumulator in TMEM)
+//                          online softmax in the exp2 domain: row max, P = exp2(S c - m), row sum
+//                          O += P V   (tcgen05.mma, M = 128, N = 64; O stays in TMEM and is
+//                          rescaled only when a row's running max grows by more than 2^8)
+// The two halves share every K/V tile and alternate on the tensor pipe, so the exponentials of
+// one half overlap the MMAs of the other.  Key tiles of range B are visited by a half only where
+// they meet the segments of its rows, and inside a tile a warp evaluates only the 32-column chunks
+// that meet the segments of its 32 rows.  The scatter back to the original token order is fused
+// into the epilogue (each thread stores its 128-byte row at the row's original position).
 #include <cuda_bf16.h>
 
 #include "mate_internal.h"
@@ -24,18 +29,40 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 128;
-constexpr int kRowBytes = 128;               // 64 bf16
+constexpr int kSoftmaxWarps = 8;
+constexpr int kMmaWarp = 8;
+constexpr int kLoadWarp0 = 9;
+constexpr int kLoadWarps = 3;
+constexpr int kLoadThreads = 32 * kLoadWarps;
+constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
+constexpr int kStages = 3;                   // K/V ring
+constexpr int kLag = 2;                      // loader: copy groups in flight behind the newest one
+
+constexpr int kRowBytes = 128;                 // 64 bf16
 constexpr int kTileBytes = kTile * kRowBytes;  // 16 KB: 128 rows
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffK = kTileBytes;
-constexpr uint32_t kOffV = 2 * kTileBytes;   // two stages
-constexpr uint32_t kOffP = 4 * kTileBytes;   // 128 x 128 bf16 = two 64-column blocks of 16 KB
-constexpr uint32_t kOffBar = 6 * kTileBytes;
-constexpr uint32_t kSmemBytes = kOffBar + 64 + 1024;  // + slack for the 1024-byte alignment
-constexpr uint32_t kTmemCols = 256;          // S: columns [0,128), O: columns [128,192)
-constexpr uint32_t kWaitLimit = 1u << 24;    // polls before a wait gives up
+constexpr uint32_t kOffQ = 0;                                // [2 buffers][2 halves] x 16 KB
+constexpr uint32_t kOffKV = 4 * kTileBytes;                  // [kStages] x (K 16 KB, V 16 KB)
+constexpr uint32_t kOffP = kOffKV + kStages * 2 * kTileBytes;  // [2 halves] x 32 KB (two 64-column blocks)
+constexpr uint32_t kOffBar = kOffP + 4 * kTileBytes;
+constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;        // + slack for the 1024-byte alignment
+constexpr uint32_t kTmemCols = 512;          // S: [0,128) half 0, [128,256) half 1; O: [256,320), [320,384)
+constexpr uint32_t kTmemO = 256;
+constexpr uint32_t kWaitLimit = 1u << 22;    // polls before a wait gives up
 constexpr float kRescaleThreshold = 8.f;     // log2 units
+
+// barrier slots (8 bytes each) behind kOffBar
+enum {
+    kBarQFull = 0,    // [2] loader -> MMA         (count: loader warps)
+    kBarQEmpty = 2,   // [2] MMA commit -> loader  (count 1)
+    kBarKVFull = 4,   // [kStages] loader -> MMA   (count: loader warps)
+    kBarKVEmpty = 8,  // [kStages] MMA -> loader   (count 2: one per half)
+    kBarSFull = 12,   // [2] MMA commit -> softmax (count 1)
+    kBarPFull = 14,   // [2] softmax -> MMA        (count 4: one per warp)
+    kBarOFull = 16,   // [2] MMA commit -> softmax (count 1)
+    kBarFinal = 18,
+    kNumBars = 19
+};
+static_assert(kStages <= 4, "barrier slots");
 
 struct Params {
     const __nv_bfloat16 *Q, *K, *V;
@@ -44,50 +71,103 @@ struct Params {
     ViewPlan rowv, colv;
     const uint8_t *head_view;
     const FwdUnit *units;
-    int n_units, N, H;
+    const int32_t *cta_begin;
+    int N, H;
     float scale_log2;  // scale * log2(e)
     int32_t *status;
+    int32_t *counters;
+    uint8_t *ws;
 };
 
-// Gathers `n_rows` rows (128 B each) of src[(row0 + i)-th view position] into a swizzled tile;
-// rows at or beyond `n_load` are zero-filled.  8 threads fetch one row, 16 rows per pass.
-__device__ __forceinline__ void load_tile(uint32_t s_tile, const __nv_bfloat16 *src_bh,
-                                          const int32_t *perm, int row0, int n_load, int n_rows,
-                                          int row_clamp, int tid) {
-    const int chunk = tid & 7;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int rr = (tid >> 3) + 16 * i;
-        if (rr < n_rows) {
-            const bool on = rr < n_load;
-            const int t = row0 + min(rr, row_clamp);
-            const int src_row = on ? perm[t] : 0;
-            const void *src = src_bh + (size_t)src_row * 64 + chunk * 8;
-            cp_async16(s_tile + rr * kRowBytes + ((chunk ^ (rr & 7)) << 4), src, on ? 16u : 0u);
-        }
+struct TileInfo {
+    int k0, w;    // first key and number of keys (<= 128)
+    bool is_b;
+};
+
+__device__ __forceinline__ int n_tiles_a(const FwdUnit &u) {
+    return u.kA_end > u.kA0 ? (u.kA_end - u.kA0 + kTile - 1) / kTile : 0;
+}
+__device__ __forceinline__ int n_tiles_b(const FwdUnit &u) {
+    return u.kB_end > u.kB0 ? (u.kB_end - u.kB0 + kTile - 1) / kTile : 0;
+}
+__device__ __forceinline__ TileInfo tile_info(const FwdUnit &u, int i, int nA) {
+    TileInfo t;
+    if (i < nA) {
+        t.k0 = u.kA0 + i * kTile;
+        t.w = min(kTile, u.kA_end - t.k0);
+        t.is_b = false;
+    } else {
+        t.k0 = u.kB0 + (i - nA) * kTile;
+        t.w = min(kTile, u.kB_end - t.k0);
+        t.is_b = true;
+    }
+    return t;
+}
+__device__ __forceinline__ int rows_of_half(const FwdUnit &u, int h) {
+    return max(0, min(kTile, u.nq - h * kTile));
+}
+// Columns [c0, c1) of the tile (multiples of 16) that half h needs; c1 <= c0 when it skips the tile.
+__device__ __forceinline__ void half_cols(const FwdUnit &u, int h, const TileInfo &t, int &c0, int &c1) {
+    if (!t.is_b) {
+        c0 = 0;
+        c1 = (t.w + 15) & ~15;
+    } else {
+        c0 = (max(u.lo[h], t.k0) - t.k0) & ~15;
+        c1 = (min(u.hi[h], t.k0 + t.w) - t.k0 + 15) & ~15;
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 2) tc_fwd_kernel(const Params p) {
+__device__ __forceinline__ FwdUnit load_unit(const FwdUnit *p) {
+    FwdUnit u;
+    const int4 *s = reinterpret_cast<const int4 *>(p);
+    int4 *d = reinterpret_cast<int4 *>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) d[i] = __ldg(s + i);
+    return u;
+}
+
+// Gathers `n_rows` rows (128 B each) into a swizzled tile: row rr comes from view position
+// row0 + min(rr, clamp) of the (example, head) slice src_bh.  8 threads fetch one row.
+__device__ __forceinline__ void load_rows(uint32_t s_tile, const __nv_bfloat16 *src_bh,
+                                          const int32_t *perm, int row0, int n_rows, int clamp,
+                                          int ltid) {
+    const int chunk = ltid & 7;
+#pragma unroll 4
+    for (int rr = ltid >> 3; rr < n_rows; rr += kLoadThreads / 8) {
+        const int src_row = perm[row0 + min(rr, clamp)];
+        const void *src = src_bh + (size_t)src_row * 64 + chunk * 8;
+        cp_async16(s_tile + rr * kRowBytes + ((chunk ^ (rr & 7)) << 4), src, 16u);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *sm = smem_raw + (base - raw);
-    const uint32_t sQ = base + kOffQ, sK = base + kOffK, sP = base + kOffP;
-    const uint32_t bar_s = base + kOffBar, bar_pv = bar_s + 8;
-    volatile uint32_t *tmem_slot = (volatile uint32_t *)(sm + kOffBar + 16);
-    volatile int *s_abort = (volatile int *)(sm + kOffBar + 20);
-    int *s_red = (int *)(sm + kOffBar + 32);  // [0..3] lo max per warp, [4..7] hi min per warp
+    const uint32_t bars = base + kOffBar;
+    volatile uint32_t *tmem_slot = (volatile uint32_t *)(sm + kOffBar + 8 * kNumBars);
+    volatile int *s_abort = (volatile int *)(sm + kOffBar + 8 * kNumBars + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     if (tid == 0) {
-        mbar_init(bar_s, 1);
-        mbar_init(bar_pv, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bars + 8 * (kBarQFull + i), kLoadWarps);
+            mbar_init(bars + 8 * (kBarQEmpty + i), 1);
+            mbar_init(bars + 8 * (kBarSFull + i), 1);
+            mbar_init(bars + 8 * (kBarPFull + i), 4);
+            mbar_init(bars + 8 * (kBarOFull + i), 1);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(bars + 8 * (kBarKVFull + i), kLoadWarps);
+            mbar_init(bars + 8 * (kBarKVEmpty + i), 2);
+        }
+        mbar_init(bars + 8 * kBarFinal, 1);
         *s_abort = 0;
         fence_mbar_init();
     }
-    if (warp == 0) {
+    if (warp == kMmaWarp) {
         tmem_alloc(smem_u32((const void *)tmem_slot), kTmemCols);
         tmem_relinquish();
     }
@@ -95,272 +175,464 @@ __global__ void __launch_bounds__(kThreads, 2) tc_fwd_kernel(const Params p) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    const uint32_t tS = tmem + ((uint32_t)(warp * 32) << 16);  // this warp's 32 lanes
-    const uint32_t tO = tS + 128;
-    uint32_t phase_s = 0, phase_pv = 0;
 
-    auto wait = [&](uint32_t bar, uint32_t parity) {
-        if (*s_abort) return;
-        if (!mbar_wait_bounded(bar, parity, kWaitLimit)) {
-            *s_abort = 1;
-            atomicOr(p.status + 1, 1);
+    // every wait is bounded; the first one to expire raises the abort flag, which ends all roles
+    auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+        for (uint32_t it = 0; it < kWaitLimit; ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((it & 63u) == 63u && *s_abort) return false;
         }
+        *s_abort = 1;
+        atomicOr(p.status + 1, 1);
+        return false;
     };
 
-    for (int u = blockIdx.x; u < p.n_units; u += gridDim.x) {
-        const FwdUnit un = p.units[u];
-        const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
-        const int32_t *perm = vp.perm + (size_t)un.b * p.N;
-        const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
-        const __nv_bfloat16 *Qbh = p.Q + bh * 64, *Kbh = p.K + bh * 64, *Vbh = p.V + bh * 64;
-        const int n_tiles = un.kA_n + un.kB_n;
-        const bool row_valid = tid < un.nq;
-        const int t_row = un.q0 + min(tid, un.nq - 1);  // rows past nq shadow the last valid row
-        const int orig = perm[t_row];
+    const int u_begin = p.cta_begin[blockIdx.x], u_end = p.cta_begin[blockIdx.x + 1];
 
-        if (n_tiles == 0) {  // padding rows: O = 0, LSE = -inf
-            if (row_valid) {
-                uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
+    if (warp < kSoftmaxWarps) {
+        // ------------------------------------------------------------------ softmax + epilogue
+        const int h = warp >> 2;
+        const int r = tid & 127;  // row of the half; TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_base + h * kTile;
+        const uint32_t tO = tmem + lane_base + kTmemO + h * 64;
+        const uint32_t sP = base + kOffP + h * 2 * kTileBytes;
+        const uint32_t bar_s = bars + 8 * (kBarSFull + h), bar_p = bars + 8 * (kBarPFull + h),
+                       bar_o = bars + 8 * (kBarOFull + h);
+        uint32_t ph_s = 0, ph_o = 0;
+        bool alive = true;
+
+        for (int u = u_begin; u < u_end && alive; ++u) {
+            const FwdUnit un = load_unit(p.units + u);
+            const int rows_h = rows_of_half(un, h);
+            if (rows_h == 0) continue;
+            const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
+            const int32_t *perm = vp.perm + (size_t)un.b * p.N;
+            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const bool row_valid = r < rows_h;
+            const int t_row = un.q0 + h * kTile + min(r, rows_h - 1);  // rows past the end shadow the last one
+            const int orig = perm[t_row];
+            const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
+
+            if (n_tiles == 0) {  // padding rows: O = 0, LSE = -inf
+                if (row_valid) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
 #pragma unroll
-                for (int c = 0; c < 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
-                p.LSE[bh + orig] = -INFINITY;
+                    for (int c = 0; c < 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
+                    p.LSE[bh + orig] = -INFINITY;
+                }
+                continue;
             }
-            continue;
-        }
 
-        const int my_lo = vp.seg_lo[(size_t)un.b * p.N + t_row];
-        const int my_hi = vp.seg_hi[(size_t)un.b * p.N + t_row];
-        {   // block-wide max of lo and min of hi: decides which B tiles need no mask
-            int lo_max = my_lo, hi_min = my_hi;
+            int my_lo = 0, my_hi = 0, w_lo_min = 0, w_lo_max = 0, w_hi_min = 0, w_hi_max = 0;
+            if (nB > 0) {
+                my_lo = vp.seg_lo[(size_t)un.b * p.N + t_row];
+                my_hi = vp.seg_hi[(size_t)un.b * p.N + t_row];
+                w_lo_min = w_lo_max = my_lo;
+                w_hi_min = w_hi_max = my_hi;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                lo_max = max(lo_max, __shfl_xor_sync(0xffffffffu, lo_max, o));
-                hi_min = min(hi_min, __shfl_xor_sync(0xffffffffu, hi_min, o));
+                for (int o = 16; o > 0; o >>= 1) {
+                    w_lo_min = min(w_lo_min, __shfl_xor_sync(0xffffffffu, w_lo_min, o));
+                    w_lo_max = max(w_lo_max, __shfl_xor_sync(0xffffffffu, w_lo_max, o));
+                    w_hi_min = min(w_hi_min, __shfl_xor_sync(0xffffffffu, w_hi_min, o));
+                    w_hi_max = max(w_hi_max, __shfl_xor_sync(0xffffffffu, w_hi_max, o));
+                }
             }
-            if (lane == 0) {
-                s_red[warp] = lo_max;
-                s_red[4 + warp] = hi_min;
-            }
-        }
 
-        auto tile_range = [&](int i, int &k0, int &w) {
-            if (i < un.kA_n) {
-                k0 = i * kTile;
-                w = min(kTile, un.kA_end - k0);
+            float m2 = -INFINITY, l = 0.f;  // running max (log2 domain, scaled) and row sum
+            bool first = true;
+
+            for (int i = 0; i < n_tiles && alive; ++i) {
+                const TileInfo t = tile_info(un, i, nA);
+                int c0, c1;
+                half_cols(un, h, t, c0, c1);
+                if (c1 <= c0) continue;
+
+                // this row's columns [r_lo, r_hi) and the warp's envelope, tile-local
+                int r_lo, r_hi, e_lo_min, e_lo_max, e_hi_min, e_hi_max;
+                if (!t.is_b) {
+                    r_lo = e_lo_min = e_lo_max = 0;
+                    r_hi = e_hi_min = e_hi_max = un.kA_end - t.k0;
+                } else {
+                    r_lo = my_lo - t.k0;
+                    r_hi = my_hi - t.k0;
+                    e_lo_min = w_lo_min - t.k0;
+                    e_lo_max = w_lo_max - t.k0;
+                    e_hi_min = w_hi_min - t.k0;
+                    e_hi_max = w_hi_max - t.k0;
+                }
+                const uint32_t r_span = (uint32_t)max(r_hi - r_lo, 0);
+                const int ch0 = c0 >> 5, ch1 = (c1 + 31) >> 5;
+
+                if (!(alive = wait(bar_s, ph_s))) break;
+                ph_s ^= 1;
+                tc_fence_after();
+
+                // pass 1: row max of the raw scores
+                float tmax = -INFINITY;
+#pragma unroll 1
+                for (int ch = ch0; ch < ch1; ++ch) {
+                    const int cb = ch * 32;
+                    if (cb + 32 <= e_lo_min || cb >= e_hi_max) continue;  // no row of the warp has keys here
+                    uint32_t v[32];
+                    tmem_ld32(tS + cb, v);
+                    tc_wait_ld();
+                    if (cb >= e_lo_max && cb + 32 <= e_hi_min) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(v[e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            const bool ok = (uint32_t)(cb + e - r_lo) < r_span;
+                            tmax = fmaxf(tmax, ok ? __uint_as_float(v[e]) : -INFINITY);
+                        }
+                    }
+                }
+                const float t2 = tmax * p.scale_log2;
+                const bool grow = t2 > m2 + kRescaleThreshold;  // also true for the first finite max
+                float alpha = 1.f;
+                if (grow) {
+                    alpha = ex2(m2 - t2);  // 0 when m2 = -inf
+                    m2 = t2;
+                    l *= alpha;
+                }
+                if (!first && __any_sync(0xffffffffu, grow)) {
+                    // the P V of the previous tile completed before S of this tile was signalled
+#pragma unroll
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c2 * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tmem_st32(tO + c2 * 32, o);
+                    }
+                    tc_wait_st();
+                }
+                const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
+
+                // pass 2: P = exp2(s * scale_log2 - m), row sum, bf16 P into swizzled shared memory
+                float lsum = 0.f;
+#pragma unroll 1
+                for (int ch = ch0; ch < ch1; ++ch) {
+                    const int cb = ch * 32;
+                    uint32_t packed[16];
+                    if (cb + 32 <= e_lo_min || cb >= e_hi_max) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) packed[e] = 0u;
+                    } else {
+                        uint32_t v[32];
+                        tmem_ld32(tS + cb, v);
+                        tc_wait_ld();
+                        const bool full = cb >= e_lo_max && cb + 32 <= e_hi_min;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            float x0 = fmaf(__uint_as_float(v[e]), p.scale_log2, neg_m);
+                            float x1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2, neg_m);
+                            if (!full) {
+                                if ((uint32_t)(cb + e - r_lo) >= r_span) x0 = -INFINITY;
+                                if ((uint32_t)(cb + e + 1 - r_lo) >= r_span) x1 = -INFINITY;
+                            }
+                            const float p0 = ex2(x0), p1 = ex2(x1);
+                            lsum += p0 + p1;
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                            packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int c8 = ch * 4 + q;  // 16-byte chunk (8 keys) of the P row
+                        const uint32_t addr = sP + (c8 >> 3) * kTileBytes + r * kRowBytes +
+                                              (((c8 & 7) ^ (r & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr),
+                                     "r"(packed[4 * q]), "r"(packed[4 * q + 1]), "r"(packed[4 * q + 2]),
+                                     "r"(packed[4 * q + 3])
+                                     : "memory");
+                    }
+                }
+                l += lsum;
+                first = false;
+
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p);
+            }
+            if (!alive) break;
+
+            // epilogue: wait for the last P V of this half
+            if (!(alive = wait(bar_o, ph_o))) break;
+            ph_o ^= 1;
+            tc_fence_after();
+            uint32_t o0[32], o1[32];
+            tmem_ld32(tO, o0);
+            tmem_ld32(tO + 32, o1);
+            tc_wait_ld();
+
+            if (un.n_parts == 1) {
+                const float inv_l = 1.f / l;
+                if (row_valid) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint32_t *src = c < 4 ? o0 + 8 * c : o1 + 8 * (c - 4);
+                        uint32_t wv[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(src[2 * e]) * inv_l,
+                                                                      __uint_as_float(src[2 * e + 1]) * inv_l);
+                            wv[e] = *reinterpret_cast<uint32_t *>(&b2);
+                        }
+                        dst[c] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                    }
+                    p.LSE[bh + orig] = (m2 + log2f(l)) * 0.6931471805599453f;
+                }
             } else {
-                k0 = un.kB0 + (i - un.kA_n) * kTile;
-                w = min(kTile, un.kB_end - k0);
+                // split unit: publish the un-normalised partial, the last part to arrive combines
+                float *part = reinterpret_cast<float *>(p.ws + ((size_t)un.ws_off << 10));
+                const int prow = h * kTile + r;
+                float4 *po = reinterpret_cast<float4 *>(part + (size_t)prow * 64);
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    po[c] = make_float4(__uint_as_float(o0[4 * c]), __uint_as_float(o0[4 * c + 1]),
+                                        __uint_as_float(o0[4 * c + 2]), __uint_as_float(o0[4 * c + 3]));
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    po[8 + c] = make_float4(__uint_as_float(o1[4 * c]), __uint_as_float(o1[4 * c + 1]),
+                                            __uint_as_float(o1[4 * c + 2]), __uint_as_float(o1[4 * c + 3]));
+                part[kUnitRows * 64 + prow] = m2;
+                part[kUnitRows * 64 + kUnitRows + prow] = l;
+                // every warp owns its 32 rows: publish, count the arrival, and the warp that comes
+                // last for these rows combines all parts (no wait on another CTA anywhere)
+                __threadfence();
+                __syncwarp();
+                int last = 0;
+                if (lane == 0) {
+                    int32_t *ctr = p.counters + 8 * un.ctr + 4 * h + (warp & 3);
+                    last = atomicAdd(ctr, 1) == un.n_parts - 1;
+                    if (last) *ctr = 0;  // ready for the next launch
+                }
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    __threadfence();
+                    const float *first_part = reinterpret_cast<const float *>(
+                        p.ws + ((size_t)(un.ws_off - un.part * (int)(kPartialBytes >> 10)) << 10));
+                    const size_t stride = kPartialBytes / sizeof(float);
+                    float M = -INFINITY;
+                    for (int q = 0; q < un.n_parts; ++q)
+                        M = fmaxf(M, __ldcg(first_part + q * stride + kUnitRows * 64 + prow));
+                    float L = 0.f, acc[64];
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) acc[e] = 0.f;
+                    for (int q = 0; q < un.n_parts; ++q) {
+                        const float *pp = first_part + q * stride;
+                        const float mq = __ldcg(pp + kUnitRows * 64 + prow);
+                        const float wq = ex2(mq - M);
+                        L = fmaf(__ldcg(pp + kUnitRows * 64 + kUnitRows + prow), wq, L);
+                        const float4 *src = reinterpret_cast<const float4 *>(pp + (size_t)prow * 64);
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const float4 x = __ldcg(src + c);
+                            acc[4 * c] = fmaf(x.x, wq, acc[4 * c]);
+                            acc[4 * c + 1] = fmaf(x.y, wq, acc[4 * c + 1]);
+                            acc[4 * c + 2] = fmaf(x.z, wq, acc[4 * c + 2]);
+                            acc[4 * c + 3] = fmaf(x.w, wq, acc[4 * c + 3]);
+                        }
+                    }
+                    const float inv_l = 1.f / L;
+                    if (row_valid) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            uint32_t wv[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[8 * c + 2 * e] * inv_l,
+                                                                          acc[8 * c + 2 * e + 1] * inv_l);
+                                wv[e] = *reinterpret_cast<uint32_t *>(&b2);
+                            }
+                            dst[c] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                        }
+                        p.LSE[bh + orig] = (M + log2f(L)) * 0.6931471805599453f;
+                    }
+                }
+            }
+            tc_fence_before();  // O was read; the next unit's first P V may overwrite it
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            uint32_t kv_cnt = 0, unit_cnt = 0, ph_p[2] = {0, 0};
+            bool alive = true;
+            const uint32_t idesc_pv = idesc_bf16(128, 64, 0, 1);
+
+            for (int u = u_begin; u < u_end && alive; ++u) {
+                const FwdUnit un = load_unit(p.units + u);
+                const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
+                if (n_tiles == 0) continue;
+                const int qb = unit_cnt & 1;
+                if (!(alive = wait(bars + 8 * (kBarQFull + qb), (unit_cnt >> 1) & 1))) break;
+                tc_fence_after();
+                const uint32_t sQ = base + kOffQ + qb * 2 * kTileBytes;
+
+                int pend_c0[2] = {0, 0}, pend_c1[2] = {0, 0}, pend_stage[2] = {0, 0};
+                bool pending[2] = {false, false}, acc[2] = {false, false};
+                const bool has_rows[2] = {rows_of_half(un, 0) > 0, rows_of_half(un, 1) > 0};
+
+                auto issue_pv = [&](int h) -> bool {
+                    if (!wait(bars + 8 * (kBarPFull + h), ph_p[h])) return false;
+                    ph_p[h] ^= 1;
+                    tc_fence_after();
+                    const uint32_t sP = base + kOffP + h * 2 * kTileBytes;
+                    const uint32_t sV = base + kOffKV + pend_stage[h] * 2 * kTileBytes + kTileBytes;
+                    const int ks0 = pend_c0[h] >> 4, ks1 = pend_c1[h] >> 4;
+                    for (int ks = ks0; ks < ks1; ++ks)
+                        mma_bf16_ss(tmem + kTmemO + h * 64,
+                                    smem_desc_sw128(sP + (ks >> 2) * kTileBytes + (ks & 3) * 32),
+                                    smem_desc_sw128(sV + ks * 16 * kRowBytes), idesc_pv, acc[h] || ks > ks0);
+                    acc[h] = true;
+                    pending[h] = false;
+                    mma_commit(bars + 8 * (kBarKVEmpty + pend_stage[h]));
+                    return true;
+                };
+
+                for (int i = 0; i < n_tiles && alive; ++i) {
+                    const TileInfo t = tile_info(un, i, nA);
+                    const int stage = kv_cnt % kStages;
+                    if (!(alive = wait(bars + 8 * (kBarKVFull + stage), (kv_cnt / kStages) & 1))) break;
+                    tc_fence_after();
+                    const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
+                    for (int h = 0; h < 2 && alive; ++h) {
+                        int c0 = 0, c1 = 0;
+                        if (has_rows[h]) half_cols(un, h, t, c0, c1);
+                        if (c1 <= c0) {  // this half skips the tile
+                            // its last P V must not keep an older stage of the ring busy meanwhile
+                            if (pending[h] && !(alive = issue_pv(h))) break;
+                            mbar_arrive(bars + 8 * (kBarKVEmpty + stage));
+                            continue;
+                        }
+                        if (pending[h] && !(alive = issue_pv(h))) break;
+                        const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            mma_bf16_ss(tmem + h * kTile + c0, smem_desc_sw128(sQ + h * kTileBytes + ks * 32),
+                                        smem_desc_sw128(sK + c0 * kRowBytes + ks * 32), idesc, ks > 0);
+                        mma_commit(bars + 8 * (kBarSFull + h));
+                        pending[h] = true;
+                        pend_c0[h] = c0;
+                        pend_c1[h] = c1;
+                        pend_stage[h] = stage;
+                    }
+                    ++kv_cnt;
+                }
+                for (int h = 0; h < 2 && alive; ++h) {
+                    if (!has_rows[h]) continue;
+                    if (pending[h] && !(alive = issue_pv(h))) break;
+                    mma_commit(bars + 8 * (kBarOFull + h));
+                }
+                if (!alive) break;
+                mma_commit(bars + 8 * (kBarQEmpty + qb));
+                ++unit_cnt;
+            }
+            // nothing of this CTA may still run on the tensor pipe when TMEM is freed
+            mma_commit(bars + 8 * kBarFinal);
+            mbar_wait_bounded(bars + 8 * kBarFinal, 0, kWaitLimit);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ loaders
+        const int ltid = tid - 32 * kLoadWarp0;
+        uint32_t kv_cnt = 0, unit_cnt = 0;
+        uint32_t pend[kLag];
+#pragma unroll
+        for (int i = 0; i < kLag; ++i) pend[i] = 0;
+        bool alive = true;
+
+        // Commits the copies issued so far as one group and signals the barrier of the group that
+        // was committed kLag groups earlier (its copies have landed by then).
+        auto commit_and_signal = [&](uint32_t bar) {
+            cp_async_commit();
+            const uint32_t oldest = pend[0];
+#pragma unroll
+            for (int i = 0; i + 1 < kLag; ++i) pend[i] = pend[i + 1];
+            pend[kLag - 1] = bar;
+            if (oldest) {
+                cp_async_wait_group<kLag>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(oldest);
             }
         };
-
-        // prologue: Q tile and key tile 0
-        load_tile(sQ, Qbh, perm, un.q0, kTile, kTile, un.nq - 1, tid);
-        {
-            int k0, w;
-            tile_range(0, k0, w);
-            const int n16 = (w + 15) & ~15;
-            load_tile(sK, Kbh, perm, k0, w, n16, kTile, tid);
-            load_tile(base + kOffV, Vbh, perm, k0, w, n16, kTile, tid);
-        }
-        cp_async_commit();
-
-        float m2 = -INFINITY, l = 0.f;  // running max (log2 domain, scaled) and row sum
-
-        for (int i = 0; i < n_tiles; ++i) {
-            const int st = i & 1;
-            int k0, w;
-            tile_range(i, k0, w);
-            const int n16 = (w + 15) & ~15;
-            const uint32_t sV = base + kOffV + st * kTileBytes;
-
-            cp_async_wait_all();
+        // Signals every group still pending.  Called before this warp blocks on a buffer that is
+        // not free yet: the consumers may need exactly those groups to free it.
+        auto flush = [&]() {
+            cp_async_wait_group<0>();
             fence_proxy_async();
-            tc_fence_before();
-            __syncthreads();  // tile i (and Q) landed; previous TMEM reads are done
-
-            if (tid == 0) {
-                tc_fence_after();
-                const uint32_t idesc = idesc_bf16(128, n16, 0, 0);
+            __syncwarp();
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    mma_bf16_ss(tmem, smem_desc_sw128(sQ + ks * 32), smem_desc_sw128(sK + ks * 32),
-                                idesc, ks > 0);
-                mma_commit(bar_s);
+            for (int i = 0; i < kLag; ++i) {
+                if (pend[i] && lane == 0) mbar_arrive(pend[i]);
+                pend[i] = 0;
             }
-            if (i > 0) {  // P V of the previous tile done: P, the other V stage and O are free
-                wait(bar_pv, phase_pv);
-                phase_pv ^= 1;
-            }
-            wait(bar_s, phase_s);
-            phase_s ^= 1;
-            tc_fence_after();
+        };
+        auto wait_free = [&](uint32_t bar, uint32_t parity) -> bool {
+            if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+            flush();
+            return wait(bar, parity);
+        };
 
-            if (i + 1 < n_tiles) {  // prefetch the next key tile while this one is in softmax
-                int k0n, wn;
-                tile_range(i + 1, k0n, wn);
-                const int n16n = (wn + 15) & ~15;
-                load_tile(sK, Kbh, perm, k0n, wn, n16n, kTile, tid);
-                load_tile(base + kOffV + (st ^ 1) * kTileBytes, Vbh, perm, k0n, wn, n16n, kTile, tid);
-                cp_async_commit();
-            }
+        for (int u = u_begin; u < u_end && alive; ++u) {
+            const FwdUnit un = load_unit(p.units + u);
+            const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
+            if (n_tiles == 0) continue;
+            const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
+            const int32_t *perm = vp.perm + (size_t)un.b * p.N;
+            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const __nv_bfloat16 *Qbh = p.Q + bh * 64, *Kbh = p.K + bh * 64, *Vbh = p.V + bh * 64;
 
-            // column window of this row inside the tile: key j = k0 + c counts iff c_lo <= c < c_hi
-            int c_lo, c_hi;
-            bool full;
-            if (i < un.kA_n) {
-                c_lo = 0;
-                c_hi = un.kA_end - k0;
-                full = (w == kTile);
-            } else {
-                c_lo = my_lo - k0;
-                c_hi = my_hi - k0;
-                const int lo_max = max(max(s_red[0], s_red[1]), max(s_red[2], s_red[3]));
-                const int hi_min = min(min(s_red[4], s_red[5]), min(s_red[6], s_red[7]));
-                full = (w == kTile) && (k0 >= lo_max) && (k0 + kTile <= hi_min);
+            const int qb = unit_cnt & 1;
+            if (!(alive = wait_free(bars + 8 * (kBarQEmpty + qb), ((unit_cnt >> 1) & 1) ^ 1))) break;
+            for (int h = 0; h < 2; ++h) {
+                const int rows_h = rows_of_half(un, h);
+                if (rows_h > 0)
+                    load_rows(base + kOffQ + (qb * 2 + h) * kTileBytes, Qbh, perm, un.q0 + h * kTile, kTile,
+                              rows_h - 1, ltid);
             }
-            const uint32_t c_span = (uint32_t)max(c_hi - c_lo, 0);
-            const int n_chunks = (n16 + 31) >> 5;
+            commit_and_signal(bars + 8 * (kBarQFull + qb));
+            ++unit_cnt;
 
-            // pass 1: row max of the raw scores
-            float tmax = -INFINITY;
-#pragma unroll 1
-            for (int ch = 0; ch < n_chunks; ++ch) {
-                uint32_t v[32];
-                tmem_ld32(tS + ch * 32, v);
-                tc_wait_ld();
-                if (full) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(v[e]));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const bool ok = (uint32_t)(ch * 32 + e - c_lo) < c_span;
-                        tmax = fmaxf(tmax, ok ? __uint_as_float(v[e]) : -INFINITY);
-                    }
-                }
-            }
-            const float t2 = tmax * p.scale_log2;
-            const bool grow = t2 > m2 + kRescaleThreshold;  // also true for the first finite max
-            float alpha = 1.f;
-            if (grow) {
-                alpha = ex2(m2 - t2);  // 0 when m2 = -inf
-                m2 = t2;
-                l *= alpha;
-            }
-            if (i > 0 && __any_sync(0xffffffffu, grow)) {
-#pragma unroll
-                for (int c2 = 0; c2 < 2; ++c2) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c2 * 32, o);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                    tmem_st32(tO + c2 * 32, o);
-                }
-                tc_wait_st();
-            }
-            const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
-
-            // pass 2: P = exp2(s * scale_log2 - m), row sum, bf16 P into swizzled shared memory
-            float lsum = 0.f;
-#pragma unroll 1
-            for (int ch = 0; ch < n_chunks; ++ch) {
-                uint32_t v[32];
-                tmem_ld32(tS + ch * 32, v);
-                tc_wait_ld();
-                uint32_t packed[16];
-#pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float x0 = fmaf(__uint_as_float(v[e]), p.scale_log2, neg_m);
-                    float x1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2, neg_m);
-                    if (!full) {
-                        if ((uint32_t)(ch * 32 + e - c_lo) >= c_span) x0 = -INFINITY;
-                        if ((uint32_t)(ch * 32 + e + 1 - c_lo) >= c_span) x1 = -INFINITY;
-                    }
-                    const float p0 = ex2(x0), p1 = ex2(x1);
-                    lsum += p0 + p1;
-                    __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                    packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
-                }
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int c8 = ch * 4 + q;  // 16-byte chunk (8 keys) of the P row
-                    const uint32_t addr = sP + (c8 >> 3) * kTileBytes + tid * kRowBytes +
-                                          (((c8 & 7) ^ (tid & 7)) << 4);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr),
-                                 "r"(packed[4 * q]), "r"(packed[4 * q + 1]), "r"(packed[4 * q + 2]),
-                                 "r"(packed[4 * q + 3])
-                                 : "memory");
-                }
-            }
-            l += lsum;
-
-            fence_proxy_async();
-            tc_fence_before();
-            __syncthreads();  // P written, S reads and O rescale finished
-
-            if (tid == 0) {
-                tc_fence_after();
-                const uint32_t idesc = idesc_bf16(128, 64, 0, 1);
-                const int n_ks = n16 >> 4;
-                for (int ks = 0; ks < n_ks; ++ks)
-                    mma_bf16_ss(tmem + 128, smem_desc_sw128(sP + (ks >> 2) * kTileBytes + (ks & 3) * 32),
-                                smem_desc_sw128(sV + ks * 16 * kRowBytes), idesc, (i > 0) || (ks > 0));
-                mma_commit(bar_pv);
+            for (int i = 0; i < n_tiles; ++i) {
+                const TileInfo t = tile_info(un, i, nA);
+                const int stage = kv_cnt % kStages;
+                if (!(alive = wait_free(bars + 8 * (kBarKVEmpty + stage), ((kv_cnt / kStages) & 1) ^ 1))) break;
+                const int n16 = (t.w + 15) & ~15;
+                const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
+                load_rows(sK, Kbh, perm, t.k0, n16, t.w - 1, ltid);
+                load_rows(sK + kTileBytes, Vbh, perm, t.k0, n16, t.w - 1, ltid);
+                commit_and_signal(bars + 8 * (kBarKVFull + stage));
+                ++kv_cnt;
             }
         }
-
-        // epilogue: O / l -> bf16, stored at the row's original position (scatter), LSE
-        wait(bar_pv, phase_pv);
-        phase_pv ^= 1;
-        tc_fence_after();
-        const float inv_l = 1.f / l;
-        uint32_t outw[32];
-#pragma unroll
-        for (int c2 = 0; c2 < 2; ++c2) {
-            uint32_t o[32];
-            tmem_ld32(tO + c2 * 32, o);
-            tc_wait_ld();
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-                __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[e]) * inv_l,
-                                                          __uint_as_float(o[e + 1]) * inv_l);
-                outw[c2 * 16 + (e >> 1)] = *reinterpret_cast<uint32_t *>(&b2);
-            }
-        }
-        if (row_valid) {
-            uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                dst[c] = make_uint4(outw[4 * c], outw[4 * c + 1], outw[4 * c + 2], outw[4 * c + 3]);
-            p.LSE[bh + orig] = (m2 + log2f(l)) * 0.6931471805599453f;
-        }
+        flush();  // drain: signal the groups still pending
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
-int g_num_sms = 0;
 bool g_attr_set = false;
 
 }  // namespace
 
 bool tc_supported(int d, int dtype) { return d == 64 && dtype == MATE_BF16; }
 
-size_t tc_fwd_workspace(const mate_plan_t *, int) { return 0; }
+size_t tc_fwd_workspace(const mate_plan_t *plan, int) { return plan->fwd_ws_bytes; }
 
 int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, float scale, void *O,
-           float *LSE, void *, cudaStream_t stream) {
+           float *LSE, void *workspace, cudaStream_t stream) {
     if (!(scale > 0.f)) return MATE_ERR_UNSUPPORTED;  // the row max is taken before scaling
     if (plan->n_fwd_units == 0) return MATE_OK;
-    if (g_num_sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return MATE_ERR_CUDA;
-    }
     if (!g_attr_set) {
         if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kSmemBytes) != cudaSuccess)
@@ -377,13 +649,14 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.colv = plan->view[1];
     p.head_view = plan->head_view_dev;
     p.units = plan->fwd_units_dev;
-    p.n_units = plan->n_fwd_units;
+    p.cta_begin = plan->fwd_cta_begin_dev;
     p.N = plan->N;
     p.H = plan->H;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = plan->status_dev;
-    const int grid = plan->n_fwd_units < 2 * g_num_sms ? plan->n_fwd_units : 2 * g_num_sms;
-    tc_fwd_kernel<<<grid, kThreads, kSmemBytes, stream>>>(p);
+    p.counters = plan->fwd_counters_dev;
+    p.ws = (uint8_t *)workspace;
+    tc_fwd_kernel<<<plan->n_ctas, kThreads, kSmemBytes, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 

@@ -9,26 +9,32 @@
 
 namespace mate {
 
-constexpr int kTile = 128;  // query rows and key columns per tile of the tensor-core kernels
+constexpr int kTile = 128;       // key columns per tile and query rows per half of a unit
+constexpr int kUnitRows = 256;   // query rows per unit of the tensor-core kernels (two halves)
 
-// One unit of forward work for the tensor-core kernel: up to 128 consecutive query rows (view
-// order) of one (example, head) and the key tiles they visit.  Key tiles are up to 128 wide.
-//   range A = keys [0, kA_end): the prefix block for table rows (kA_end = P), every valid key for
-//             prefix rows (kA_end = n_valid).  Inside it a key j counts iff j < kA_end.
-//   range B = keys [kB0, kB_end): the union of the segments the query rows belong to (table rows
-//             only, kB0 >= P).  Inside it key j counts for a row iff seg_lo[row] <= j < seg_hi[row].
+// One unit of work of the tensor-core forward: up to 256 consecutive query rows (view order) of one
+// (example, head) -- half 0 = the first 128 rows, half 1 = the rest -- and the key tiles (128 wide)
+// they visit, in this order:
+//   range A = keys [kA0, kA_end): the prefix block for table rows ([0, P)), a slice of all valid
+//             keys for prefix rows.  Key j counts for every row iff j < kA_end.
+//   range B = keys [kB0, kB_end): the union of the segments the rows belong to (table rows only).
+//             Key j counts for a row iff seg_lo[row] <= j < seg_hi[row]; half h touches only the
+//             tiles that meet [lo[h], hi[h]) (min seg_lo / max seg_hi over its rows).
+// Prefix rows whose key range is long are split along the keys into n_parts units; each writes an
+// un-normalised partial result to the workspace at ws_off (KiB); per group of 32 rows the part
+// that finishes last (counted in counters[8 * ctr + row / 32]) combines them.
 struct FwdUnit {
     int32_t b, h;
-    int32_t q0, nq;        // first query row (view order) and number of rows (<= 128)
-    int32_t kA_end, kA_n;  // range A: end key and number of 128-key tiles
-    int32_t kB0, kB_end;   // range B: first and end key
-    int32_t kB_n;          // range B: number of tiles
-    int32_t part, n_parts; // split-key bookkeeping: this unit is part `part` of `n_parts`
-    int32_t slot;          // partial-result slot in the workspace when n_parts > 1, else -1
-    int32_t cost;          // key tiles visited (sort key, largest first)
-    int32_t pad_[3];
+    int32_t q0, nq;
+    int32_t kA0, kA_end;
+    int32_t kB0, kB_end;
+    int32_t lo[2], hi[2];
+    int32_t n_parts, part;
+    int32_t ws_off, ctr;
 };
 static_assert(sizeof(FwdUnit) == 64, "FwdUnit is read as four 16-byte words");
+// bytes of one partial result: 256 rows x (64 fp32 + running max + row sum)
+constexpr size_t kPartialBytes = (size_t)kUnitRows * (64 + 2) * sizeof(float);
 
 struct ViewPlan {
     int32_t *perm = nullptr;      // [B, N]   view position -> original position
@@ -53,14 +59,17 @@ struct mate_plan_s {
     std::vector<int64_t> pairs;          // [B, 2] unmasked pairs per example and view
     int32_t *status_dev = nullptr;       // device status word(s): [0] = id validation, [1] = kernel timeouts
     void *dev_block = nullptr;           // one allocation backing all device arrays above
-    // tensor-core forward work-list
+    void *work_block = nullptr;          // one allocation backing the work-lists below
+    // tensor-core forward work-list: units grouped by CTA (cost-balanced at plan time)
     mate::FwdUnit *fwd_units_dev = nullptr;
+    int32_t *fwd_cta_begin_dev = nullptr; // [n_ctas + 1] first unit of every CTA
+    int32_t *fwd_counters_dev = nullptr;  // [8 * n_fwd_slots] arrival counters of split units (self-resetting)
     int n_fwd_units = 0;
-    int n_fwd_slots = 0;                 // partial-result slots (split prefix rows)
-    std::vector<mate::FwdUnit> fwd_units; // host copy (combine pass bookkeeping)
-    mate::FwdUnit *bwd_units_dev = nullptr;
-    int n_bwd_units = 0;
-    int n_bwd_slots = 0;
+    int n_fwd_slots = 0;                  // split units (prefix rows cut along the keys)
+    int n_ctas = 0;                       // CTAs the work-list was balanced for (SMs of the plan's device)
+    size_t fwd_ws_bytes = 0;              // partial results of the split units
+    std::vector<mate::FwdUnit> fwd_units; // host copy
+    std::vector<int32_t> fwd_cta_begin;   // host copy
 };
 
 namespace mate {
