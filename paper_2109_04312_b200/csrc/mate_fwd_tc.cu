@@ -126,17 +126,29 @@ __device__ __forceinline__ FwdUnit load_unit(const FwdUnit *p) {
     return u;
 }
 
-// Gathers `n_rows` rows (128 B each) into a swizzled tile: row rr comes from view position
-// row0 + min(rr, clamp) of the (example, head) slice src_bh.  8 threads fetch one row.
-__device__ __forceinline__ void load_rows(uint32_t s_tile, const __nv_bfloat16 *src_bh,
-                                          const int32_t *perm, int row0, int n_rows, int clamp,
-                                          int ltid) {
+// The loaders copy a tile of up to 128 rows (128 B each) in passes of kRowsPerPass rows, 8 threads
+// per row.  Row rr of the tile comes from view position row0 + min(rr, clamp); its original
+// position is looked up first for every pass (independent loads), then the 16-byte copies follow.
+constexpr int kRowsPerPass = kLoadThreads / 8;
+constexpr int kPasses = (kTile + kRowsPerPass - 1) / kRowsPerPass;
+
+__device__ __forceinline__ void load_indices(int (&idx)[kPasses], const int32_t *perm, int row0,
+                                             int n_rows, int clamp, int ltid) {
+#pragma unroll
+    for (int i = 0; i < kPasses; ++i) {
+        const int rr = (ltid >> 3) + kRowsPerPass * i;
+        idx[i] = rr < n_rows ? __ldg(perm + row0 + min(rr, clamp)) : -1;
+    }
+}
+__device__ __forceinline__ void copy_rows(uint32_t s_tile, const __nv_bfloat16 *src_bh,
+                                          const int (&idx)[kPasses], int ltid) {
     const int chunk = ltid & 7;
-#pragma unroll 4
-    for (int rr = ltid >> 3; rr < n_rows; rr += kLoadThreads / 8) {
-        const int src_row = perm[row0 + min(rr, clamp)];
-        const void *src = src_bh + (size_t)src_row * 64 + chunk * 8;
-        cp_async16(s_tile + rr * kRowBytes + ((chunk ^ (rr & 7)) << 4), src, 16u);
+#pragma unroll
+    for (int i = 0; i < kPasses; ++i) {
+        const int rr = (ltid >> 3) + kRowsPerPass * i;
+        if (idx[i] >= 0)
+            cp_async16(s_tile + rr * kRowBytes + ((chunk ^ (rr & 7)) << 4),
+                       src_bh + (size_t)idx[i] * 64 + chunk * 8, 16u);
     }
 }
 
@@ -269,7 +281,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 tc_fence_after();
 
                 // pass 1: row max of the raw scores
-                float tmax = -INFINITY;
+                float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
                 for (int ch = ch0; ch < ch1; ++ch) {
                     const int cb = ch * 32;
@@ -279,15 +291,21 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     tc_wait_ld();
                     if (cb >= e_lo_max && cb + 32 <= e_hi_min) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) tmax = fmaxf(tmax, __uint_as_float(v[e]));
+                        for (int e = 0; e < 32; e += 8) {
+                            tm[0] = fmax3(tm[0], __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                            tm[1] = fmax3(tm[1], __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                            tm[2] = fmax3(tm[2], __uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+                            tm[3] = fmax3(tm[3], __uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
+                        }
                     } else {
 #pragma unroll
                         for (int e = 0; e < 32; ++e) {
                             const bool ok = (uint32_t)(cb + e - r_lo) < r_span;
-                            tmax = fmaxf(tmax, ok ? __uint_as_float(v[e]) : -INFINITY);
+                            tm[e & 3] = fmaxf(tm[e & 3], ok ? __uint_as_float(v[e]) : -INFINITY);
                         }
                     }
                 }
+                const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
                 const float t2 = tmax * p.scale_log2;
                 const bool grow = t2 > m2 + kRescaleThreshold;  // also true for the first finite max
                 float alpha = 1.f;
@@ -312,7 +330,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
 
                 // pass 2: P = exp2(s * scale_log2 - m), row sum, bf16 P into swizzled shared memory
-                float lsum = 0.f;
+                float lsum = 0.f, lsum1 = 0.f;
 #pragma unroll 1
                 for (int ch = ch0; ch < ch1; ++ch) {
                     const int cb = ch * 32;
@@ -334,7 +352,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                                 if ((uint32_t)(cb + e + 1 - r_lo) >= r_span) x1 = -INFINITY;
                             }
                             const float p0 = ex2(x0), p1 = ex2(x1);
-                            lsum += p0 + p1;
+                            lsum += p0;
+                            lsum1 += p1;
                             __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
                             packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
                         }
@@ -350,7 +369,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                                      : "memory");
                     }
                 }
-                l += lsum;
+                l += lsum + lsum1;
                 first = false;
 
                 fence_proxy_async();
@@ -576,7 +595,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             }
         };
         auto wait_free = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (__all_sync(0xffffffffu, mbar_try_wait(bar, parity))) return true;
+            if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
             flush();
             return wait(bar, parity);
         };
@@ -594,9 +613,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             if (!(alive = wait_free(bars + 8 * (kBarQEmpty + qb), ((unit_cnt >> 1) & 1) ^ 1))) break;
             for (int h = 0; h < 2; ++h) {
                 const int rows_h = rows_of_half(un, h);
-                if (rows_h > 0)
-                    load_rows(base + kOffQ + (qb * 2 + h) * kTileBytes, Qbh, perm, un.q0 + h * kTile, kTile,
-                              rows_h - 1, ltid);
+                if (rows_h > 0) {
+                    int idx[kPasses];
+                    load_indices(idx, perm, un.q0 + h * kTile, kTile, rows_h - 1, ltid);
+                    copy_rows(base + kOffQ + (qb * 2 + h) * kTileBytes, Qbh, idx, ltid);
+                }
             }
             commit_and_signal(bars + 8 * (kBarQFull + qb));
             ++unit_cnt;
@@ -604,11 +625,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             for (int i = 0; i < n_tiles; ++i) {
                 const TileInfo t = tile_info(un, i, nA);
                 const int stage = kv_cnt % kStages;
+                int idx[kPasses];
+                load_indices(idx, perm, t.k0, (t.w + 15) & ~15, t.w - 1, ltid);
                 if (!(alive = wait_free(bars + 8 * (kBarKVEmpty + stage), ((kv_cnt / kStages) & 1) ^ 1))) break;
-                const int n16 = (t.w + 15) & ~15;
                 const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
-                load_rows(sK, Kbh, perm, t.k0, n16, t.w - 1, ltid);
-                load_rows(sK + kTileBytes, Vbh, perm, t.k0, n16, t.w - 1, ltid);
+                copy_rows(sK, Kbh, idx, ltid);
+                copy_rows(sK + kTileBytes, Vbh, idx, ltid);
                 commit_and_signal(bars + 8 * (kBarKVFull + stage));
                 ++kv_cnt;
             }
