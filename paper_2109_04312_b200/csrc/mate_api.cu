@@ -166,55 +166,36 @@ int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
             }
         }
         if (pass == 0) {
-            // a split part should cost about a quarter of a CTA's share (never below two key tiles)
+            // a split part should cost about half of a CTA's share (never below two key tiles)
             const int64_t share = total / std::max(pl->n_ctas, 1);
-            const int64_t part_cost = std::max<int64_t>(share / 4, 1);
+            const int64_t part_cost = std::max<int64_t>(share / 2, 1);
             // cost of one key tile of a full prefix unit: 8 warps x 4 chunks
             split_tiles = std::max<int64_t>(2, part_cost / 32);
         }
     }
     static_assert(mate::kPartialBytes % 1024 == 0, "ws_off counts KiB");
 
-    // longest first, each to the least loaded CTA
+    // longest first: the CTAs of the persistent kernel take units from the head of this list as
+    // they become free (a shared counter), so the order is the whole schedule
     std::stable_sort(all.begin(), all.end(), [](const UnitCost &a, const UnitCost &b) { return a.cost > b.cost; });
     const int n_ctas = std::max(pl->n_ctas, 1);
-    std::vector<std::vector<int>> mine(n_ctas);
-    std::vector<std::pair<int64_t, int>> heap;  // (load, cta) min-heap
-    for (int c = 0; c < n_ctas; ++c) heap.push_back({0, c});
-    auto cmp = [](const std::pair<int64_t, int> &a, const std::pair<int64_t, int> &b) { return a > b; };
-    std::make_heap(heap.begin(), heap.end(), cmp);
-    for (int i = 0; i < (int)all.size(); ++i) {
-        std::pop_heap(heap.begin(), heap.end(), cmp);
-        auto &top = heap.back();
-        mine[top.second].push_back(i);
-        top.first += all[i].cost;
-        std::push_heap(heap.begin(), heap.end(), cmp);
-    }
     pl->fwd_units.clear();
-    pl->fwd_cta_begin.assign(n_ctas + 1, 0);
-    for (int c = 0; c < n_ctas; ++c) {
-        pl->fwd_cta_begin[c] = (int32_t)pl->fwd_units.size();
-        for (int i : mine[c]) pl->fwd_units.push_back(all[i].u);
+    int64_t total_cost = 0;
+    for (const UnitCost &uc : all) {
+        pl->fwd_units.push_back(uc.u);
+        total_cost += uc.cost;
     }
-    pl->fwd_cta_begin[n_ctas] = (int32_t)pl->fwd_units.size();
     pl->n_fwd_units = (int)pl->fwd_units.size();
-    if (getenv("MATE_LOG")) {
-        int64_t mx = 0, sum = 0;
-        for (auto &hc : heap) {
-            mx = std::max(mx, hc.first);
-            sum += hc.first;
-        }
-        fprintf(stderr, "[mate] forward work-list: %d units, %d split slots, %d CTAs, cost max %lld mean %.1f, "
-                        "split at %lld key tiles, workspace %zu bytes\n",
-                pl->n_fwd_units, pl->n_fwd_slots, n_ctas, (long long)mx, (double)sum / n_ctas,
-                (long long)split_tiles, pl->fwd_ws_bytes);
-    }
+    if (getenv("MATE_LOG"))
+        fprintf(stderr, "[mate] forward work-list: %d units, %d split slots, %d CTAs, cost total %lld (%.1f per CTA, "
+                        "largest unit %lld), split at %lld key tiles, workspace %zu bytes\n",
+                pl->n_fwd_units, pl->n_fwd_slots, n_ctas, (long long)total_cost, (double)total_cost / n_ctas,
+                all.empty() ? 0ll : (long long)all.front().cost, (long long)split_tiles, pl->fwd_ws_bytes);
 
     // device copy: units, CTA offsets, arrival counters (zeroed once; the kernel resets them)
     Carver c(nullptr);
     c.take<FwdUnit>(pl->n_fwd_units);
-    c.take<int32_t>(n_ctas + 1);
-    c.take<int32_t>(8 * (size_t)std::max(pl->n_fwd_slots, 1));
+    c.take<int32_t>(mate::kSchedWords + 8 * (size_t)pl->n_fwd_slots);
     const size_t bytes = align_up(c.off, 256);
     if (cudaMalloc(&pl->work_block, bytes) != cudaSuccess) {
         cudaGetLastError();
@@ -222,8 +203,7 @@ int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
     }
     Carver d((char *)pl->work_block);
     pl->fwd_units_dev = d.take<FwdUnit>(pl->n_fwd_units);
-    pl->fwd_cta_begin_dev = d.take<int32_t>(n_ctas + 1);
-    pl->fwd_counters_dev = d.take<int32_t>(8 * (size_t)std::max(pl->n_fwd_slots, 1));
+    pl->fwd_counters_dev = d.take<int32_t>(mate::kSchedWords + 8 * (size_t)pl->n_fwd_slots);
     return MATE_OK;
 }
 
@@ -342,11 +322,8 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
         mate_plan_destroy(pl);
         return rc;
     }
-    bool up = cudaMemsetAsync(pl->fwd_counters_dev, 0, sizeof(int32_t) * 8 * (size_t)std::max(pl->n_fwd_slots, 1),
-                              st) == cudaSuccess;
-    up = up && cudaMemcpyAsync(pl->fwd_cta_begin_dev, pl->fwd_cta_begin.data(),
-                               sizeof(int32_t) * pl->fwd_cta_begin.size(), cudaMemcpyHostToDevice,
-                               st) == cudaSuccess;
+    bool up = cudaMemsetAsync(pl->fwd_counters_dev, 0,
+                              sizeof(int32_t) * (mate::kSchedWords + 8 * (size_t)pl->n_fwd_slots), st) == cudaSuccess;
     if (pl->n_fwd_units > 0)
         up = up && cudaMemcpyAsync(pl->fwd_units_dev, pl->fwd_units.data(), sizeof(FwdUnit) * pl->n_fwd_units,
                                    cudaMemcpyHostToDevice, st) == cudaSuccess;
@@ -389,7 +366,15 @@ int mate_plan_status(const mate_plan_t *plan, void *stream) {
         cudaMemsetAsync(plan->status_dev + 1, 0, sizeof(int32_t), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
         return MATE_ERR_CUDA;
-    return s[1] != 0 ? MATE_ERR_TIMEOUT : MATE_OK;
+    if (s[1] != 0) {
+        // a kernel that gave up may have left the scheduling and arrival counters half way
+        if (cudaMemsetAsync(plan->fwd_counters_dev, 0,
+                            sizeof(int32_t) * (mate::kSchedWords + 8 * (size_t)plan->n_fwd_slots), st) != cudaSuccess ||
+            cudaStreamSynchronize(st) != cudaSuccess)
+            return MATE_ERR_CUDA;
+        return MATE_ERR_TIMEOUT;
+    }
+    return MATE_OK;
 }
 
 static int check_common(const mate_plan_t *plan, int d, int dtype, unsigned flags, bool *use_tc) {

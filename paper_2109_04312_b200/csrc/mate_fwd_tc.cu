@@ -60,8 +60,12 @@ enum {
     kBarPFull = 14,   // [2] softmax -> MMA        (count 4: one per warp)
     kBarOFull = 16,   // [2] MMA commit -> softmax (count 1)
     kBarFinal = 18,
-    kNumBars = 19
+    kBarSchedFull = 19,   // [kSchedDepth] scheduler -> every warp that follows the unit list (count 1)
+    kBarSchedEmpty = 23,  // [kSchedDepth] those warps -> scheduler (count kSchedReaders)
+    kNumBars = 27
 };
+constexpr int kSchedDepth = 4;
+constexpr int kSchedReaders = kSoftmaxWarps + 1 + kLoadWarps;
 static_assert(kStages <= 4, "barrier slots");
 
 struct Params {
@@ -71,7 +75,7 @@ struct Params {
     ViewPlan rowv, colv;
     const uint8_t *head_view;
     const FwdUnit *units;
-    const int32_t *cta_begin;
+    int n_units;
     int N, H;
     float scale_log2;  // scale * log2(e)
     int32_t *status;
@@ -160,6 +164,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     const uint32_t bars = base + kOffBar;
     volatile uint32_t *tmem_slot = (volatile uint32_t *)(sm + kOffBar + 8 * kNumBars);
     volatile int *s_abort = (volatile int *)(sm + kOffBar + 8 * kNumBars + 4);
+    volatile int *s_unit = (volatile int *)(sm + kOffBar + 8 * kNumBars + 8);  // [kSchedDepth] unit ids
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -174,6 +179,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         for (int i = 0; i < kStages; ++i) {
             mbar_init(bars + 8 * (kBarKVFull + i), kLoadWarps);
             mbar_init(bars + 8 * (kBarKVEmpty + i), 2);
+        }
+        for (int i = 0; i < kSchedDepth; ++i) {
+            mbar_init(bars + 8 * (kBarSchedFull + i), 1);
+            mbar_init(bars + 8 * (kBarSchedEmpty + i), kSchedReaders);
         }
         mbar_init(bars + 8 * kBarFinal, 1);
         *s_abort = 0;
@@ -199,7 +208,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         return false;
     };
 
-    const int u_begin = p.cta_begin[blockIdx.x], u_end = p.cta_begin[blockIdx.x + 1];
+    // The unit list is shared by all CTAs: lane 0 of the first loader warp takes the next index from
+    // a global counter and publishes it in a small ring; every warp that follows the list reads the
+    // n-th entry here (-1 = the list is exhausted) and frees the slot for the scheduler.
+    auto next_unit = [&](uint32_t n) -> int {
+        const int slot = n % kSchedDepth;
+        if (!wait(bars + 8 * (kBarSchedFull + slot), (n / kSchedDepth) & 1)) return -1;
+        const int u = s_unit[slot];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8 * (kBarSchedEmpty + slot));
+        return u;
+    };
 
     if (warp < kSoftmaxWarps) {
         // ------------------------------------------------------------------ softmax + epilogue
@@ -214,7 +233,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         uint32_t ph_s = 0, ph_o = 0;
         bool alive = true;
 
-        for (int u = u_begin; u < u_end && alive; ++u) {
+        for (uint32_t n = 0; alive; ++n) {
+            const int u = next_unit(n);
+            if (u < 0) break;
             const FwdUnit un = load_unit(p.units + u);
             const int rows_h = rows_of_half(un, h);
             if (rows_h == 0) continue;
@@ -427,53 +448,51 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 __syncwarp();
                 int last = 0;
                 if (lane == 0) {
-                    int32_t *ctr = p.counters + 8 * un.ctr + 4 * h + (warp & 3);
+                    int32_t *ctr = p.counters + kSchedWords + 8 * un.ctr + 4 * h + (warp & 3);
                     last = atomicAdd(ctr, 1) == un.n_parts - 1;
                     if (last) *ctr = 0;  // ready for the next launch
                 }
                 last = __shfl_sync(0xffffffffu, last, 0);
                 if (last) {
+                    // The warp combines its 32 rows one row at a time with all lanes on the row's 64
+                    // columns (two per lane), so every load of a partial row is one coalesced 256-byte
+                    // request; a row's weights live in the lane of that row and travel by shuffle.
                     __threadfence();
                     const float *first_part = reinterpret_cast<const float *>(
                         p.ws + ((size_t)(un.ws_off - un.part * (int)(kPartialBytes >> 10)) << 10));
                     const size_t stride = kPartialBytes / sizeof(float);
+                    const float *ml = first_part + kUnitRows * 64 + prow;  // this lane's row: max, then sum
                     float M = -INFINITY;
+                    for (int q = 0; q < un.n_parts; ++q) M = fmaxf(M, __ldcg(ml + q * stride));
+                    float L = 0.f;
                     for (int q = 0; q < un.n_parts; ++q)
-                        M = fmaxf(M, __ldcg(first_part + q * stride + kUnitRows * 64 + prow));
-                    float L = 0.f, acc[64];
+                        L = fmaf(__ldcg(ml + q * stride + kUnitRows), ex2(__ldcg(ml + q * stride) - M), L);
+                    const float inv_L = 1.f / L;
+                    float2 acc[32];
 #pragma unroll
-                    for (int e = 0; e < 64; ++e) acc[e] = 0.f;
+                    for (int rr = 0; rr < 32; ++rr) acc[rr] = make_float2(0.f, 0.f);
+                    const int row0 = h * kTile + (warp & 3) * 32;  // first row of this warp in the partials
                     for (int q = 0; q < un.n_parts; ++q) {
-                        const float *pp = first_part + q * stride;
-                        const float mq = __ldcg(pp + kUnitRows * 64 + prow);
-                        const float wq = ex2(mq - M);
-                        L = fmaf(__ldcg(pp + kUnitRows * 64 + kUnitRows + prow), wq, L);
-                        const float4 *src = reinterpret_cast<const float4 *>(pp + (size_t)prow * 64);
+                        const float wq = ex2(__ldcg(ml + q * stride) - M) * inv_L;
+                        const float2 *src = reinterpret_cast<const float2 *>(first_part + q * stride + (size_t)row0 * 64) + lane;
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) {
-                            const float4 x = __ldcg(src + c);
-                            acc[4 * c] = fmaf(x.x, wq, acc[4 * c]);
-                            acc[4 * c + 1] = fmaf(x.y, wq, acc[4 * c + 1]);
-                            acc[4 * c + 2] = fmaf(x.z, wq, acc[4 * c + 2]);
-                            acc[4 * c + 3] = fmaf(x.w, wq, acc[4 * c + 3]);
+                        for (int rr = 0; rr < 32; ++rr) {
+                            const float2 x = __ldcg(src + rr * 32);
+                            const float w = __shfl_sync(0xffffffffu, wq, rr);
+                            acc[rr].x = fmaf(x.x, w, acc[rr].x);
+                            acc[rr].y = fmaf(x.y, w, acc[rr].y);
                         }
                     }
-                    const float inv_l = 1.f / L;
-                    if (row_valid) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            uint32_t wv[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[8 * c + 2 * e] * inv_l,
-                                                                          acc[8 * c + 2 * e + 1] * inv_l);
-                                wv[e] = *reinterpret_cast<uint32_t *>(&b2);
-                            }
-                            dst[c] = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                    for (int rr = 0; rr < 32; ++rr) {
+                        const int dst_row = __shfl_sync(0xffffffffu, orig, rr);
+                        const bool ok = __shfl_sync(0xffffffffu, (int)row_valid, rr) != 0;
+                        if (ok) {
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(acc[rr].x, acc[rr].y);
+                            reinterpret_cast<__nv_bfloat162 *>(p.O + (bh + dst_row) * 64)[lane] = b2;
                         }
-                        p.LSE[bh + orig] = (M + log2f(L)) * 0.6931471805599453f;
                     }
+                    if (row_valid) p.LSE[bh + orig] = (M + log2f(L)) * 0.6931471805599453f;
                 }
             }
             tc_fence_before();  // O was read; the next unit's first P V may overwrite it
@@ -485,7 +504,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             bool alive = true;
             const uint32_t idesc_pv = idesc_bf16(128, 64, 0, 1);
 
-            for (int u = u_begin; u < u_end && alive; ++u) {
+            for (uint32_t n = 0; alive; ++n) {
+                const int slot = n % kSchedDepth;
+                if (!(alive = wait(bars + 8 * (kBarSchedFull + slot), (n / kSchedDepth) & 1))) break;
+                const int u = s_unit[slot];
+                mbar_arrive(bars + 8 * (kBarSchedEmpty + slot));
+                if (u < 0) break;
                 const FwdUnit un = load_unit(p.units + u);
                 const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
                 if (n_tiles == 0) continue;
@@ -600,7 +624,51 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             return wait(bar, parity);
         };
 
-        for (int u = u_begin; u < u_end && alive; ++u) {
+        // scheduler state (lane 0 of the first loader warp only)
+        uint32_t produced = 0;
+        bool list_done = false;
+        auto produce = [&]() -> bool {  // publishes one more entry; false = gave up
+            const int slot = produced % kSchedDepth;
+            if (produced >= (uint32_t)kSchedDepth) {
+                const uint32_t par = ((produced / kSchedDepth) & 1) ^ 1;
+                const uint32_t bar = bars + 8 * (kBarSchedEmpty + slot);
+                if (!wait(bar, par)) return false;
+            }
+            // the first unit of a CTA is its own index; later ones come from the shared counter
+            const int u = produced == 0 ? (int)blockIdx.x : atomicAdd(p.counters, 1) + (int)gridDim.x;
+            const int val = u < p.n_units ? u : -1;
+            s_unit[slot] = val;
+            mbar_arrive(bars + 8 * (kBarSchedFull + slot));  // release: the store above is visible to the readers
+            ++produced;
+            if (val < 0) list_done = true;
+            return true;
+        };
+
+        for (uint32_t n = 0; alive; ++n) {
+            // Entry n is taken only now, when the loaders are about to start on it (they run a few key
+            // tiles ahead of the other warps): taking units earlier would hand them out before it is
+            // known which CTA becomes free first.  Before a loader warp blocks here it signals its
+            // pending copy groups: the warps it would wait for may need exactly those tiles.
+            {
+                const int slot = n % kSchedDepth;
+                bool must_wait;
+                if (warp == kLoadWarp0) {  // the scheduler's warp: blocks only if the ring slot is still being read
+                    must_wait = produced >= (uint32_t)kSchedDepth &&
+                                !mbar_test_wait(bars + 8 * (kBarSchedEmpty + slot), ((produced / kSchedDepth) & 1) ^ 1);
+                    must_wait = __shfl_sync(0xffffffffu, (int)must_wait, 0) != 0;
+                } else {
+                    must_wait = !__all_sync(0xffffffffu, mbar_test_wait(bars + 8 * (kBarSchedFull + slot),
+                                                                       (n / kSchedDepth) & 1));
+                }
+                if (must_wait) flush();
+            }
+            if (ltid == 0) {
+                while (!list_done && produced <= n)
+                    if (!produce()) break;
+            }
+            __syncwarp();
+            const int u = next_unit(n);
+            if (u < 0) break;
             const FwdUnit un = load_unit(p.units + u);
             const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
             if (n_tiles == 0) continue;
@@ -641,6 +709,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
+    if (tid == 0) {
+        // the CTA that finishes last puts the scheduling counters back to zero for the next launch
+        // (every CTA has taken its last index by the time it counts itself as finished)
+        __threadfence();
+        if (atomicAdd(p.counters + 1, 1) == (int)gridDim.x - 1) {
+            p.counters[0] = 0;
+            p.counters[1] = 0;
+        }
+    }
 }
 
 bool g_attr_set = false;
@@ -671,7 +748,7 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.colv = plan->view[1];
     p.head_view = plan->head_view_dev;
     p.units = plan->fwd_units_dev;
-    p.cta_begin = plan->fwd_cta_begin_dev;
+    p.n_units = plan->n_fwd_units;
     p.N = plan->N;
     p.H = plan->H;
     p.scale_log2 = scale * 1.4426950408889634f;

@@ -10,6 +10,7 @@
 namespace mate {
 
 constexpr int kTile = 128;       // key columns per tile and query rows per half of a unit
+constexpr int kSchedWords = 8;   // scheduling counters in front of the split-unit counters
 constexpr int kUnitRows = 256;   // query rows per unit of the tensor-core kernels (two halves)
 
 // One unit of work of the tensor-core forward: up to 256 consecutive query rows (view order) of one
@@ -22,7 +23,7 @@ constexpr int kUnitRows = 256;   // query rows per unit of the tensor-core kerne
 //             tiles that meet [lo[h], hi[h]) (min seg_lo / max seg_hi over its rows).
 // Prefix rows whose key range is long are split along the keys into n_parts units; each writes an
 // un-normalised partial result to the workspace at ws_off (KiB); per group of 32 rows the part
-// that finishes last (counted in counters[8 * ctr + row / 32]) combines them.
+// that finishes last (counted in counters[kSchedWords + 8 * ctr + row / 32]) combines them.
 struct FwdUnit {
     int32_t b, h;
     int32_t q0, nq;
@@ -60,16 +61,18 @@ struct mate_plan_s {
     int32_t *status_dev = nullptr;       // device status word(s): [0] = id validation, [1] = kernel timeouts
     void *dev_block = nullptr;           // one allocation backing all device arrays above
     void *work_block = nullptr;          // one allocation backing the work-lists below
-    // tensor-core forward work-list: units grouped by CTA (cost-balanced at plan time)
+    // tensor-core forward work-list: units by decreasing cost; the CTAs of the persistent kernel
+    // take them in this order through a shared counter
     mate::FwdUnit *fwd_units_dev = nullptr;
-    int32_t *fwd_cta_begin_dev = nullptr; // [n_ctas + 1] first unit of every CTA
-    int32_t *fwd_counters_dev = nullptr;  // [8 * n_fwd_slots] arrival counters of split units (self-resetting)
+    // [kSchedWords + 8 * n_fwd_slots]: [0] next unit, [1] CTAs finished, then the arrival counters of
+    // the split units.  Zero between launches (the kernel resets what it counted), which is why
+    // two forward calls on one plan must not overlap on the GPU.
+    int32_t *fwd_counters_dev = nullptr;
     int n_fwd_units = 0;
     int n_fwd_slots = 0;                  // split units (prefix rows cut along the keys)
-    int n_ctas = 0;                       // CTAs the work-list was balanced for (SMs of the plan's device)
+    int n_ctas = 0;                       // CTAs of the persistent kernel (SMs of the plan's device)
     size_t fwd_ws_bytes = 0;              // partial results of the split units
     std::vector<mate::FwdUnit> fwd_units; // host copy
-    std::vector<int32_t> fwd_cta_begin;   // host copy
 };
 
 namespace mate {
