@@ -48,6 +48,7 @@ constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;        // + slack for the 
 constexpr uint32_t kTmemCols = 512;          // S: [0,128) half 0, [128,256) half 1; O: [256,320), [320,384)
 constexpr uint32_t kTmemO = 256;
 constexpr uint32_t kWaitLimit = 1u << 22;    // polls before a wait gives up
+constexpr uint32_t kSpinLimit = 1u << 26;    // rounds without progress before the MMA issuer gives up
 constexpr float kRescaleThreshold = 8.f;     // log2 units
 
 // barrier slots (8 bytes each) behind kOffBar
@@ -227,7 +228,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + h * kTile;
         const uint32_t tO = tmem + lane_base + kTmemO + h * 64;
-        const uint32_t sP = base + kOffP + h * 2 * kTileBytes;
         const uint32_t bar_s = bars + 8 * (kBarSFull + h), bar_p = bars + 8 * (kBarPFull + h),
                        bar_o = bars + 8 * (kBarOFull + h);
         uint32_t ph_s = 0, ph_o = 0;
@@ -379,21 +379,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                             packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
                         }
                     }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int c8 = ch * 4 + q;  // 16-byte chunk (8 keys) of the P row
-                        const uint32_t addr = sP + (c8 >> 3) * kTileBytes + r * kRowBytes +
-                                              (((c8 & 7) ^ (r & 7)) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr),
-                                     "r"(packed[4 * q]), "r"(packed[4 * q + 1]), "r"(packed[4 * q + 2]),
-                                     "r"(packed[4 * q + 3])
-                                     : "memory");
-                    }
+                    tmem_st16(tS + ch * 16, packed);  // P (bf16 pairs) over the S columns already consumed
                 }
                 l += lsum + lsum1;
                 first = false;
 
-                fence_proxy_async();
+                tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p);
@@ -518,61 +509,88 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 tc_fence_after();
                 const uint32_t sQ = base + kOffQ + qb * 2 * kTileBytes;
 
-                int pend_c0[2] = {0, 0}, pend_c1[2] = {0, 0}, pend_stage[2] = {0, 0};
+                // Each half walks the key tiles of the unit on its own and is served as soon as what
+                // it waits for is there (its P for the next P V, the next K/V tile for the next
+                // Q K^T), so a half never idles behind the other one.  A tile's ring stage is
+                // released by both halves: by the commit behind the P V, or at once by a half that
+                // skips the tile -- but only while the tile occupies the stage, hence tile by tile.
+                int cur[2] = {0, 0};                 // next tile this half has to look at
+                int last_t[2] = {-1, -1};            // last tile the half takes part in
+                int pend_c0[2] = {0, 0}, pend_c1[2] = {0, 0}, pend_stage[2] = {0, 0}, pend_tile[2] = {0, 0};
                 bool pending[2] = {false, false}, acc[2] = {false, false};
-                const bool has_rows[2] = {rows_of_half(un, 0) > 0, rows_of_half(un, 1) > 0};
-
-                auto issue_pv = [&](int h) -> bool {
-                    if (!wait(bars + 8 * (kBarPFull + h), ph_p[h])) return false;
-                    ph_p[h] ^= 1;
-                    tc_fence_after();
-                    const uint32_t sP = base + kOffP + h * 2 * kTileBytes;
-                    const uint32_t sV = base + kOffKV + pend_stage[h] * 2 * kTileBytes + kTileBytes;
-                    const int ks0 = pend_c0[h] >> 4, ks1 = pend_c1[h] >> 4;
-                    for (int ks = ks0; ks < ks1; ++ks)
-                        mma_bf16_ss(tmem + kTmemO + h * 64,
-                                    smem_desc_sw128(sP + (ks >> 2) * kTileBytes + (ks & 3) * 32),
-                                    smem_desc_sw128(sV + ks * 16 * kRowBytes), idesc_pv, acc[h] || ks > ks0);
-                    acc[h] = true;
-                    pending[h] = false;
-                    mma_commit(bars + 8 * (kBarKVEmpty + pend_stage[h]));
-                    return true;
-                };
-
-                for (int i = 0; i < n_tiles && alive; ++i) {
-                    const TileInfo t = tile_info(un, i, nA);
-                    const int stage = kv_cnt % kStages;
-                    if (!(alive = wait(bars + 8 * (kBarKVFull + stage), (kv_cnt / kStages) & 1))) break;
-                    tc_fence_after();
-                    const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
-                    for (int h = 0; h < 2 && alive; ++h) {
-                        int c0 = 0, c1 = 0;
-                        if (has_rows[h]) half_cols(un, h, t, c0, c1);
-                        if (c1 <= c0) {  // this half skips the tile
-                            // its last P V must not keep an older stage of the ring busy meanwhile
-                            if (pending[h] && !(alive = issue_pv(h))) break;
-                            mbar_arrive(bars + 8 * (kBarKVEmpty + stage));
-                            continue;
-                        }
-                        if (pending[h] && !(alive = issue_pv(h))) break;
-                        const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            mma_bf16_ss(tmem + h * kTile + c0, smem_desc_sw128(sQ + h * kTileBytes + ks * 32),
-                                        smem_desc_sw128(sK + c0 * kRowBytes + ks * 32), idesc, ks > 0);
-                        mma_commit(bars + 8 * (kBarSFull + h));
-                        pending[h] = true;
-                        pend_c0[h] = c0;
-                        pend_c1[h] = c1;
-                        pend_stage[h] = stage;
+                for (int h = 0; h < 2; ++h) {
+                    if (rows_of_half(un, h) == 0) continue;
+                    for (int i = 0; i < n_tiles; ++i) {
+                        int c0, c1;
+                        half_cols(un, h, tile_info(un, i, nA), c0, c1);
+                        if (c1 > c0) last_t[h] = i;
                     }
-                    ++kv_cnt;
                 }
-                for (int h = 0; h < 2 && alive; ++h) {
-                    if (!has_rows[h]) continue;
-                    if (pending[h] && !(alive = issue_pv(h))) break;
-                    mma_commit(bars + 8 * (kBarOFull + h));
+                int kv_ready = 0;  // tiles of this unit known to have landed
+                uint32_t idle = 0;
+                while (alive && (cur[0] < n_tiles || cur[1] < n_tiles || pending[0] || pending[1])) {
+                    bool progress = false;
+                    if (kv_ready < n_tiles) {
+                        const uint32_t c = kv_cnt + kv_ready;
+                        if (mbar_test_wait(bars + 8 * (kBarKVFull + c % kStages), (c / kStages) & 1)) {
+                            ++kv_ready;
+                            progress = true;
+                        }
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (pending[h] && mbar_test_wait(bars + 8 * (kBarPFull + h), ph_p[h])) {
+                            ph_p[h] ^= 1;
+                            tc_fence_after();
+                            const uint32_t sV = base + kOffKV + pend_stage[h] * 2 * kTileBytes + kTileBytes;
+                            const int ks0 = pend_c0[h] >> 4, ks1 = pend_c1[h] >> 4;
+                            for (int ks = ks0; ks < ks1; ++ks)
+                                mma_bf16_ts(tmem + kTmemO + h * 64, tmem + h * kTile + ks * 8,
+                                            smem_desc_sw128(sV + ks * 16 * kRowBytes), idesc_pv, acc[h] || ks > ks0);
+                            acc[h] = true;
+                            pending[h] = false;
+                            mma_commit(bars + 8 * (kBarKVEmpty + pend_stage[h]));
+                            if (pend_tile[h] == last_t[h]) mma_commit(bars + 8 * (kBarOFull + h));
+                            progress = true;
+                        }
+                        if (!pending[h] && cur[h] < n_tiles && cur[h] < kv_ready) {
+                            const int i = cur[h]++;
+                            const TileInfo t = tile_info(un, i, nA);
+                            const int stage = (kv_cnt + i) % kStages;
+                            int c0 = 0, c1 = 0;
+                            if (last_t[h] >= 0) half_cols(un, h, t, c0, c1);
+                            if (c1 <= c0) {
+                                mbar_arrive(bars + 8 * (kBarKVEmpty + stage));  // this half skips the tile
+                            } else {
+                                tc_fence_after();
+                                const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
+                                const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks)
+                                    mma_bf16_ss(tmem + h * kTile + c0,
+                                                smem_desc_sw128(sQ + h * kTileBytes + ks * 32),
+                                                smem_desc_sw128(sK + c0 * kRowBytes + ks * 32), idesc, ks > 0);
+                                mma_commit(bars + 8 * (kBarSFull + h));
+                                pending[h] = true;
+                                pend_c0[h] = c0;
+                                pend_c1[h] = c1;
+                                pend_stage[h] = stage;
+                                pend_tile[h] = i;
+                            }
+                            progress = true;
+                        }
+                    }
+                    if (progress) {
+                        idle = 0;
+                    } else if (++idle > kSpinLimit || ((idle & 255u) == 0 && *s_abort)) {
+                        if (idle > kSpinLimit) {
+                            *s_abort = 1;
+                            atomicOr(p.status + 1, 1);
+                        }
+                        alive = false;
+                    }
                 }
+                kv_cnt += n_tiles;
                 if (!alive) break;
                 mma_commit(bars + 8 * (kBarQEmpty + qb));
                 ++unit_cnt;
