@@ -542,11 +542,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         if (pending[h] && mbar_test_wait(bars + 8 * (kBarPFull + h), ph_p[h])) {
                             ph_p[h] ^= 1;
                             tc_fence_after();
-                            const uint32_t sV = base + kOffKV + pend_stage[h] * 2 * kTileBytes + kTileBytes;
-                            const int ks0 = pend_c0[h] >> 4, ks1 = pend_c1[h] >> 4;
-                            for (int ks = ks0; ks < ks1; ++ks)
-                                mma_bf16_ts(tmem + kTmemO + h * 64, tmem + h * kTile + ks * 8,
-                                            smem_desc_sw128(sV + ks * 16 * kRowBytes), idesc_pv, acc[h] || ks > ks0);
+                            const int ks0 = pend_c0[h] >> 4, n_ks = (pend_c1[h] - pend_c0[h]) >> 4;
+                            // V rows 16 ks .. 16 ks + 15 (2 KB per step), P columns 8 ks .. 8 ks + 7
+                            uint32_t v_lo = smem_desc_lo(base + kOffKV + pend_stage[h] * 2 * kTileBytes + kTileBytes +
+                                                         ks0 * 16 * kRowBytes);
+                            uint32_t tP = tmem + h * kTile + ks0 * 8;
+                            const uint32_t tOh = tmem + kTmemO + h * 64;
+                            mma_ts_lean_flag(tOh, tP, v_lo, idesc_pv, acc[h]);
+#pragma unroll 1
+                            for (int ks = 1; ks < n_ks; ++ks) {
+                                v_lo += (16 * kRowBytes) >> 4;
+                                tP += 8;
+                                mma_ts_lean<1>(tOh, tP, v_lo, idesc_pv);
+                            }
                             acc[h] = true;
                             pending[h] = false;
                             mma_commit(bars + 8 * (kBarKVEmpty + pend_stage[h]));
@@ -563,13 +571,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                                 mbar_arrive(bars + 8 * (kBarKVEmpty + stage));  // this half skips the tile
                             } else {
                                 tc_fence_after();
-                                const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
                                 const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
-#pragma unroll
-                                for (int ks = 0; ks < 4; ++ks)
-                                    mma_bf16_ss(tmem + h * kTile + c0,
-                                                smem_desc_sw128(sQ + h * kTileBytes + ks * 32),
-                                                smem_desc_sw128(sK + c0 * kRowBytes + ks * 32), idesc, ks > 0);
+                                const uint32_t q_lo = smem_desc_lo(sQ + h * kTileBytes);
+                                const uint32_t k_lo = smem_desc_lo(base + kOffKV + stage * 2 * kTileBytes + c0 * kRowBytes);
+                                const uint32_t tSh = tmem + h * kTile + c0;
+                                mma_ss_lean<0>(tSh, q_lo, k_lo, idesc);      // K = 64 as four steps of 16 (32 bytes)
+                                mma_ss_lean<1>(tSh, q_lo + 2, k_lo + 2, idesc);
+                                mma_ss_lean<1>(tSh, q_lo + 4, k_lo + 4, idesc);
+                                mma_ss_lean<1>(tSh, q_lo + 6, k_lo + 6, idesc);
                                 mma_commit(bars + 8 * (kBarSFull + h));
                                 pending[h] = true;
                                 pend_c0[h] = c0;
