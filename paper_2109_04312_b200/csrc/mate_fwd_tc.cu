@@ -5,8 +5,8 @@
 //
 //   warps 0-3   softmax of half 0 (query rows 0..127 of the unit), one thread per row
 //   warps 4-7   softmax of half 1 (rows 128..255)
-//   warp  8     one thread issues every tcgen05.mma
-//   warps 9-11  loaders: gather Q, K, V rows by view-order index into 128-byte swizzled shared
+//   warps 8, 9  one thread each issues the tcgen05.mma of half 0 / half 1
+//   warps 10-11 loaders: gather Q, K, V rows by view-order index into 128-byte swizzled shared
 //               memory with 16-byte cp.async (the gather of Section 3.1 fused into the loads)
 //
 // Per key tile and half:   S = Q K^T  (tcgen05.mma, M = 128, N <= 128, K = 64, accumulator in TMEM)
@@ -25,14 +25,28 @@
 
 namespace mate {
 
+// Optional cycle counters (compile with -DMATE_TRACE): per CTA and role, clock64() time spent in
+// the marked regions.  Profiling aid only; compiled out of the library.
+#ifdef MATE_TRACE
+__device__ long long g_trace[148 * 32];
+#define TR_T0(var) const long long var = clock64()
+#define TR_ADD(cat, var) tr[cat] += clock64() - (var)
+#define TR_INC(cat) tr[cat] += 1
+#else
+#define TR_T0(var)
+#define TR_ADD(cat, var)
+#define TR_INC(cat)
+#endif
+
 namespace {
 
 using namespace ptx;
 
 constexpr int kSoftmaxWarps = 8;
-constexpr int kMmaWarp = 8;
-constexpr int kLoadWarp0 = 9;
-constexpr int kLoadWarps = 3;
+constexpr int kMmaWarp = 8;   // warps 8 and 9: one MMA-issuing thread per half
+constexpr int kMmaWarps = 2;
+constexpr int kLoadWarp0 = 10;
+constexpr int kLoadWarps = 2;
 constexpr int kLoadThreads = 32 * kLoadWarps;
 constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
 constexpr int kStages = 3;                   // K/V ring
@@ -45,28 +59,29 @@ constexpr uint32_t kOffKV = 4 * kTileBytes;                  // [kStages] x (K 1
 constexpr uint32_t kOffP = kOffKV + kStages * 2 * kTileBytes;  // [2 halves] x 32 KB (two 64-column blocks)
 constexpr uint32_t kOffBar = kOffP + 4 * kTileBytes;
 constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;        // + slack for the 1024-byte alignment
-constexpr uint32_t kTmemCols = 512;          // S: [0,128) half 0, [128,256) half 1; O: [256,320), [320,384)
+// tensor memory: S of half h at column 128 h; O at 256 + 64 h; P (bf16 pairs) at 384 + 64 h
+constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemO = 256;
-constexpr uint32_t kWaitLimit = 1u << 22;    // polls before a wait gives up
-constexpr uint32_t kSpinLimit = 1u << 26;    // rounds without progress before the MMA issuer gives up
+constexpr uint32_t kTmemP = 384;
+constexpr uint32_t kWaitLimit = 4096;        // tries (up to 1 ms each) before a wait gives up
 constexpr float kRescaleThreshold = 8.f;     // log2 units
 
 // barrier slots (8 bytes each) behind kOffBar
 enum {
     kBarQFull = 0,    // [2] loader -> MMA         (count: loader warps)
-    kBarQEmpty = 2,   // [2] MMA commit -> loader  (count 1)
+    kBarQEmpty = 2,   // [2] MMA commit -> loader  (count 2: one per half)
     kBarKVFull = 4,   // [kStages] loader -> MMA   (count: loader warps)
     kBarKVEmpty = 8,  // [kStages] MMA -> loader   (count 2: one per half)
     kBarSFull = 12,   // [2] MMA commit -> softmax (count 1)
     kBarPFull = 14,   // [2] softmax -> MMA        (count 4: one per warp)
-    kBarOFull = 16,   // [2] MMA commit -> softmax (count 1)
-    kBarFinal = 18,
-    kBarSchedFull = 19,   // [kSchedDepth] scheduler -> every warp that follows the unit list (count 1)
-    kBarSchedEmpty = 23,  // [kSchedDepth] those warps -> scheduler (count kSchedReaders)
-    kNumBars = 27
+    kBarPVDone = 16,  // [2] MMA commit -> softmax: the P V of a tile is complete (count 1)
+    kBarFinal = 18,       // [2]
+    kBarSchedFull = 20,   // [kSchedDepth] scheduler -> every warp that follows the unit list (count 1)
+    kBarSchedEmpty = 24,  // [kSchedDepth] those warps -> scheduler (count kSchedReaders)
+    kNumBars = 28
 };
 constexpr int kSchedDepth = 4;
-constexpr int kSchedReaders = kSoftmaxWarps + 1 + kLoadWarps;
+constexpr int kSchedReaders = kSoftmaxWarps + kMmaWarps + kLoadWarps;
 static_assert(kStages <= 4, "barrier slots");
 
 struct Params {
@@ -157,6 +172,47 @@ __device__ __forceinline__ void copy_rows(uint32_t s_tile, const __nv_bfloat16 *
     }
 }
 
+// Row max over one chunk of 32 scores (tile-local columns cb .. cb + 31); a column c counts for the
+// row iff r_lo <= c < r_lo + r_span, and `full` says that every column of the chunk counts.
+__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], int cb, bool full, int r_lo,
+                                          uint32_t r_span, float (&tm)[4]) {
+    if (full) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 8) {
+            tm[0] = fmax3(tm[0], __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+            tm[1] = fmax3(tm[1], __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+            tm[2] = fmax3(tm[2], __uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+            tm[3] = fmax3(tm[3], __uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const bool ok = (uint32_t)(cb + e - r_lo) < r_span;
+            tm[e & 3] = fmaxf(tm[e & 3], ok ? __uint_as_float(v[e]) : -INFINITY);
+        }
+    }
+}
+// P of one chunk: exp2(s * scale_log2 + neg_m) for the columns that count, 0 elsewhere, packed as
+// bf16 pairs (even column in the low half); adds the row sums of even / odd columns to l0 / l1.
+__device__ __forceinline__ void chunk_exp(const uint32_t (&v)[32], int cb, bool full, int r_lo,
+                                          uint32_t r_span, float scale_log2, float neg_m,
+                                          uint32_t (&packed)[16], float &l0, float &l1) {
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        float x0 = fmaf(__uint_as_float(v[e]), scale_log2, neg_m);
+        float x1 = fmaf(__uint_as_float(v[e + 1]), scale_log2, neg_m);
+        if (!full) {
+            if ((uint32_t)(cb + e - r_lo) >= r_span) x0 = -INFINITY;
+            if ((uint32_t)(cb + e + 1 - r_lo) >= r_span) x1 = -INFINITY;
+        }
+        const float p0 = ex2(x0), p1 = ex2(x1);
+        l0 += p0;
+        l1 += p1;
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+        packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -172,10 +228,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(bars + 8 * (kBarQFull + i), kLoadWarps);
-            mbar_init(bars + 8 * (kBarQEmpty + i), 1);
+            mbar_init(bars + 8 * (kBarQEmpty + i), 2);
             mbar_init(bars + 8 * (kBarSFull + i), 1);
             mbar_init(bars + 8 * (kBarPFull + i), 4);
-            mbar_init(bars + 8 * (kBarOFull + i), 1);
+            mbar_init(bars + 8 * (kBarPVDone + i), 1);
         }
         for (int i = 0; i < kStages; ++i) {
             mbar_init(bars + 8 * (kBarKVFull + i), kLoadWarps);
@@ -186,6 +242,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             mbar_init(bars + 8 * (kBarSchedEmpty + i), kSchedReaders);
         }
         mbar_init(bars + 8 * kBarFinal, 1);
+        mbar_init(bars + 8 * (kBarFinal + 1), 1);
         *s_abort = 0;
         fence_mbar_init();
     }
@@ -202,13 +259,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
         for (uint32_t it = 0; it < kWaitLimit; ++it) {
             if (mbar_try_wait(bar, parity)) return true;
-            if ((it & 63u) == 63u && *s_abort) return false;
+            if (*s_abort) return false;
         }
         *s_abort = 1;
         atomicOr(p.status + 1, 1);
         return false;
     };
 
+#ifdef MATE_TRACE
+    long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const long long tr_start = clock64();
+#endif
     // The unit list is shared by all CTAs: lane 0 of the first loader warp takes the next index from
     // a global counter and publishes it in a small ring; every warp that follows the list reads the
     // n-th entry here (-1 = the list is exhausted) and frees the slot for the scheduler.
@@ -228,14 +289,18 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + h * kTile;
         const uint32_t tO = tmem + lane_base + kTmemO + h * 64;
+        const uint32_t tP = tmem + lane_base + kTmemP + h * 64;
         const uint32_t bar_s = bars + 8 * (kBarSFull + h), bar_p = bars + 8 * (kBarPFull + h),
-                       bar_o = bars + 8 * (kBarOFull + h);
-        uint32_t ph_s = 0, ph_o = 0;
+                       bar_pv = bars + 8 * (kBarPVDone + h);
+        uint32_t ph_s = 0, ph_pv = 0;
         bool alive = true;
 
         for (uint32_t n = 0; alive; ++n) {
+            TR_T0(t_nu);
             const int u = next_unit(n);
+            TR_ADD(7, t_nu);
             if (u < 0) break;
+            TR_T0(t_setup);
             const FwdUnit un = load_unit(p.units + u);
             const int rows_h = rows_of_half(un, h);
             if (rows_h == 0) continue;
@@ -272,6 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 }
             }
 
+            TR_ADD(5, t_setup);
             float m2 = -INFINITY, l = 0.f;  // running max (log2 domain, scaled) and row sum
             bool first = true;
 
@@ -297,35 +363,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 const uint32_t r_span = (uint32_t)max(r_hi - r_lo, 0);
                 const int ch0 = c0 >> 5, ch1 = (c1 + 31) >> 5;
 
+                TR_T0(t_ws);
                 if (!(alive = wait(bar_s, ph_s))) break;
                 ph_s ^= 1;
                 tc_fence_after();
+                TR_ADD(0, t_ws);
+                TR_T0(t_p1);
 
-                // pass 1: row max of the raw scores
+                // pass 1: row max of the raw scores, 32 columns at a time (chunks in which no row of
+                // the warp has a key are not looked at)
                 float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
                 for (int ch = ch0; ch < ch1; ++ch) {
                     const int cb = ch * 32;
-                    if (cb + 32 <= e_lo_min || cb >= e_hi_max) continue;  // no row of the warp has keys here
+                    if (cb + 32 <= e_lo_min || cb >= e_hi_max) continue;
                     uint32_t v[32];
                     tmem_ld32(tS + cb, v);
                     tc_wait_ld();
-                    if (cb >= e_lo_max && cb + 32 <= e_hi_min) {
-#pragma unroll
-                        for (int e = 0; e < 32; e += 8) {
-                            tm[0] = fmax3(tm[0], __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
-                            tm[1] = fmax3(tm[1], __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                            tm[2] = fmax3(tm[2], __uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
-                            tm[3] = fmax3(tm[3], __uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-                        }
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const bool ok = (uint32_t)(cb + e - r_lo) < r_span;
-                            tm[e & 3] = fmaxf(tm[e & 3], ok ? __uint_as_float(v[e]) : -INFINITY);
-                        }
-                    }
+                    chunk_max(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, tm);
                 }
+                TR_ADD(2, t_p1);
                 const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
                 const float t2 = tmax * p.scale_log2;
                 const bool grow = t2 > m2 + kRescaleThreshold;  // also true for the first finite max
@@ -335,8 +392,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     m2 = t2;
                     l *= alpha;
                 }
+                // P of the previous tile is still being read, and O written, until that tile's P V is done
+                if (!first) {
+                    TR_T0(t_wpv);
+                    if (!(alive = wait(bar_pv, ph_pv))) break;
+                    ph_pv ^= 1;
+                    tc_fence_after();
+                    TR_ADD(1, t_wpv);
+                }
                 if (!first && __any_sync(0xffffffffu, grow)) {
-                    // the P V of the previous tile completed before S of this tile was signalled
 #pragma unroll
                     for (int c2 = 0; c2 < 2; ++c2) {
                         uint32_t o[32];
@@ -350,7 +414,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 }
                 const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
 
-                // pass 2: P = exp2(s * scale_log2 - m), row sum, bf16 P into swizzled shared memory
+                // pass 2: P = exp2(s * scale_log2 - m) as bf16 pairs into the P columns, row sum
+                TR_T0(t_p2);
                 float lsum = 0.f, lsum1 = 0.f;
 #pragma unroll 1
                 for (int ch = ch0; ch < ch1; ++ch) {
@@ -363,23 +428,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         uint32_t v[32];
                         tmem_ld32(tS + cb, v);
                         tc_wait_ld();
-                        const bool full = cb >= e_lo_max && cb + 32 <= e_hi_min;
-#pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            float x0 = fmaf(__uint_as_float(v[e]), p.scale_log2, neg_m);
-                            float x1 = fmaf(__uint_as_float(v[e + 1]), p.scale_log2, neg_m);
-                            if (!full) {
-                                if ((uint32_t)(cb + e - r_lo) >= r_span) x0 = -INFINITY;
-                                if ((uint32_t)(cb + e + 1 - r_lo) >= r_span) x1 = -INFINITY;
-                            }
-                            const float p0 = ex2(x0), p1 = ex2(x1);
-                            lsum += p0;
-                            lsum1 += p1;
-                            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                            packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
-                        }
+                        chunk_exp(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, p.scale_log2, neg_m,
+                                  packed, lsum, lsum1);
                     }
-                    tmem_st16(tS + ch * 16, packed);  // P (bf16 pairs) over the S columns already consumed
+                    tmem_st16(tP + ch * 16, packed);
                 }
                 l += lsum + lsum1;
                 first = false;
@@ -388,13 +440,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p);
+                TR_ADD(3, t_p2);
+                TR_INC(4);
             }
             if (!alive) break;
 
             // epilogue: wait for the last P V of this half
-            if (!(alive = wait(bar_o, ph_o))) break;
-            ph_o ^= 1;
+            TR_T0(t_ep);
+            if (!(alive = wait(bar_pv, ph_pv))) break;
+            ph_pv ^= 1;
             tc_fence_after();
+            TR_ADD(1, t_ep);
             uint32_t o0[32], o1[32];
             tmem_ld32(tO, o0);
             tmem_ld32(tO + 32, o1);
@@ -487,13 +543,22 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 }
             }
             tc_fence_before();  // O was read; the next unit's first P V may overwrite it
+            TR_ADD(6, t_ep);
         }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ MMA issuer (one thread)
+    } else if (warp < kLoadWarp0) {
+        // ------------------------------------------------------------------ MMA issuers (one thread per half)
+        // Per half: Q K^T of a tile -> (softmax) -> when P arrives, the Q K^T of the half's next tile
+        // goes first (the softmax warps wait for it) and the P V of the finished tile behind it.  A
+        // tile's ring stage is released by both halves: by the commit behind the P V, or, for a
+        // tile the half skips, by a plain arrival once the tile has landed.
         if (lane == 0) {
-            uint32_t kv_cnt = 0, unit_cnt = 0, ph_p[2] = {0, 0};
+            const int h = warp - kMmaWarp;
+            uint32_t kv_cnt = 0, unit_cnt = 0, ph_p = 0;
             bool alive = true;
             const uint32_t idesc_pv = idesc_bf16(128, 64, 0, 1);
+            const uint32_t tSh0 = tmem + h * kTile, tOh = tmem + kTmemO + h * 64, tPh0 = tmem + kTmemP + h * 64;
+            const uint32_t bar_p = bars + 8 * (kBarPFull + h), bar_s = bars + 8 * (kBarSFull + h),
+                           bar_pv = bars + 8 * (kBarPVDone + h);
 
             for (uint32_t n = 0; alive; ++n) {
                 const int slot = n % kSchedDepth;
@@ -505,99 +570,95 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
                 if (n_tiles == 0) continue;
                 const int qb = unit_cnt & 1;
+                TR_T0(t_qf);
                 if (!(alive = wait(bars + 8 * (kBarQFull + qb), (unit_cnt >> 1) & 1))) break;
                 tc_fence_after();
-                const uint32_t sQ = base + kOffQ + qb * 2 * kTileBytes;
+                TR_ADD(0, t_qf);
+                const uint32_t q_lo = smem_desc_lo(base + kOffQ + (qb * 2 + h) * kTileBytes);
+                const bool has_rows = rows_of_half(un, h) > 0;
 
-                // Each half walks the key tiles of the unit on its own and is served as soon as what
-                // it waits for is there (its P for the next P V, the next K/V tile for the next
-                // Q K^T), so a half never idles behind the other one.  A tile's ring stage is
-                // released by both halves: by the commit behind the P V, or at once by a half that
-                // skips the tile -- but only while the tile occupies the stage, hence tile by tile.
-                int cur[2] = {0, 0};                 // next tile this half has to look at
-                int last_t[2] = {-1, -1};            // last tile the half takes part in
-                int pend_c0[2] = {0, 0}, pend_c1[2] = {0, 0}, pend_stage[2] = {0, 0}, pend_tile[2] = {0, 0};
-                bool pending[2] = {false, false}, acc[2] = {false, false};
-                for (int h = 0; h < 2; ++h) {
-                    if (rows_of_half(un, h) == 0) continue;
-                    for (int i = 0; i < n_tiles; ++i) {
-                        int c0, c1;
-                        half_cols(un, h, tile_info(un, i, nA), c0, c1);
-                        if (c1 > c0) last_t[h] = i;
-                    }
-                }
-                int kv_ready = 0;  // tiles of this unit known to have landed
-                uint32_t idle = 0;
-                while (alive && (cur[0] < n_tiles || cur[1] < n_tiles || pending[0] || pending[1])) {
-                    bool progress = false;
-                    if (kv_ready < n_tiles) {
-                        const uint32_t c = kv_cnt + kv_ready;
-                        if (mbar_test_wait(bars + 8 * (kBarKVFull + c % kStages), (c / kStages) & 1)) {
-                            ++kv_ready;
-                            progress = true;
-                        }
-                    }
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (pending[h] && mbar_test_wait(bars + 8 * (kBarPFull + h), ph_p[h])) {
-                            ph_p[h] ^= 1;
-                            tc_fence_after();
-                            const int ks0 = pend_c0[h] >> 4, n_ks = (pend_c1[h] - pend_c0[h]) >> 4;
-                            // V rows 16 ks .. 16 ks + 15 (2 KB per step), P columns 8 ks .. 8 ks + 7
-                            uint32_t v_lo = smem_desc_lo(base + kOffKV + pend_stage[h] * 2 * kTileBytes + kTileBytes +
-                                                         ks0 * 16 * kRowBytes);
-                            uint32_t tP = tmem + h * kTile + ks0 * 8;
-                            const uint32_t tOh = tmem + kTmemO + h * 64;
-                            mma_ts_lean_flag(tOh, tP, v_lo, idesc_pv, acc[h]);
+                int qk_c0 = 0, qk_c1 = 0, qk_stage = 0;  // Q K^T issued, P not seen yet
+                int pv_c0 = 0, pv_c1 = 0, pv_stage = 0;  // P seen, P V not issued yet
+                bool wait_p = false, have_p = false, acc = false;
+
+                auto issue_pv = [&]() {
+                    TR_T0(t_pv);
+                    const int ks0 = pv_c0 >> 4, n_ks = (pv_c1 - pv_c0) >> 4;
+                    // V rows 16 ks .. 16 ks + 15 (2 KB per step), P columns 8 ks .. 8 ks + 7
+                    uint32_t v_lo = smem_desc_lo(base + kOffKV + pv_stage * 2 * kTileBytes + kTileBytes + ks0 * 16 * kRowBytes);
+                    uint32_t tPh = tPh0 + ks0 * 8;
+                    mma_ts_lean_flag(tOh, tPh, v_lo, idesc_pv, acc);
 #pragma unroll 1
-                            for (int ks = 1; ks < n_ks; ++ks) {
-                                v_lo += (16 * kRowBytes) >> 4;
-                                tP += 8;
-                                mma_ts_lean<1>(tOh, tP, v_lo, idesc_pv);
-                            }
-                            acc[h] = true;
-                            pending[h] = false;
-                            mma_commit(bars + 8 * (kBarKVEmpty + pend_stage[h]));
-                            if (pend_tile[h] == last_t[h]) mma_commit(bars + 8 * (kBarOFull + h));
-                            progress = true;
-                        }
-                        if (!pending[h] && cur[h] < n_tiles && cur[h] < kv_ready) {
-                            const int i = cur[h]++;
-                            const TileInfo t = tile_info(un, i, nA);
-                            const int stage = (kv_cnt + i) % kStages;
-                            int c0 = 0, c1 = 0;
-                            if (last_t[h] >= 0) half_cols(un, h, t, c0, c1);
-                            if (c1 <= c0) {
-                                mbar_arrive(bars + 8 * (kBarKVEmpty + stage));  // this half skips the tile
-                            } else {
-                                tc_fence_after();
-                                const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
-                                const uint32_t q_lo = smem_desc_lo(sQ + h * kTileBytes);
-                                const uint32_t k_lo = smem_desc_lo(base + kOffKV + stage * 2 * kTileBytes + c0 * kRowBytes);
-                                const uint32_t tSh = tmem + h * kTile + c0;
-                                mma_ss_lean<0>(tSh, q_lo, k_lo, idesc);      // K = 64 as four steps of 16 (32 bytes)
-                                mma_ss_lean<1>(tSh, q_lo + 2, k_lo + 2, idesc);
-                                mma_ss_lean<1>(tSh, q_lo + 4, k_lo + 4, idesc);
-                                mma_ss_lean<1>(tSh, q_lo + 6, k_lo + 6, idesc);
-                                mma_commit(bars + 8 * (kBarSFull + h));
-                                pending[h] = true;
-                                pend_c0[h] = c0;
-                                pend_c1[h] = c1;
-                                pend_stage[h] = stage;
-                                pend_tile[h] = i;
-                            }
-                            progress = true;
-                        }
+                    for (int ks = 1; ks < n_ks; ++ks) {
+                        v_lo += (16 * kRowBytes) >> 4;
+                        tPh += 8;
+                        mma_ts_lean<1>(tOh, tPh, v_lo, idesc_pv);
                     }
-                    if (progress) {
-                        idle = 0;
-                    } else if (++idle > kSpinLimit || ((idle & 255u) == 0 && *s_abort)) {
-                        if (idle > kSpinLimit) {
-                            *s_abort = 1;
-                            atomicOr(p.status + 1, 1);
+                    acc = true;
+                    have_p = false;
+                    mma_commit(bar_pv);
+                    mma_commit(bars + 8 * (kBarKVEmpty + pv_stage));
+                    TR_ADD(3, t_pv);
+                };
+                auto take_p = [&]() -> bool {  // waits for the P of the outstanding Q K^T
+                    TR_T0(t_wp);
+                    if (!wait(bar_p, ph_p)) return false;
+                    TR_ADD(1, t_wp);
+                    ph_p ^= 1;
+                    tc_fence_after();
+                    wait_p = false;
+                    have_p = true;
+                    pv_c0 = qk_c0;
+                    pv_c1 = qk_c1;
+                    pv_stage = qk_stage;
+                    return true;
+                };
+
+                for (int i = 0; i < n_tiles && alive; ++i) {
+                    const TileInfo t = tile_info(un, i, nA);
+                    const uint32_t c = kv_cnt + i;
+                    const int stage = c % kStages;
+                    const uint32_t bar_kv = bars + 8 * (kBarKVFull + stage), par_kv = (c / kStages) & 1;
+                    int c0 = 0, c1 = 0;
+                    if (has_rows) half_cols(un, h, t, c0, c1);
+                    if (c1 <= c0) {  // this half skips the tile
+                        if (wait_p) {  // nothing to issue ahead of the P V of the previous tile
+                            if (!(alive = take_p())) break;
+                            issue_pv();
                         }
-                        alive = false;
+                        TR_T0(t_kv);
+                        if (!(alive = wait(bar_kv, par_kv))) break;
+                        TR_ADD(5, t_kv);
+                        mbar_arrive(bars + 8 * (kBarKVEmpty + stage));
+                        continue;
                     }
+                    if (wait_p && !(alive = take_p())) break;
+                    if (have_p && !mbar_test_wait(bar_kv, par_kv)) issue_pv();  // the next tile is not there yet
+                    TR_T0(t_kv);
+                    if (!(alive = wait(bar_kv, par_kv))) break;
+                    TR_ADD(5, t_kv);
+                    tc_fence_after();
+                    {
+                        TR_T0(t_qk);
+                        const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
+                        const uint32_t k_lo = smem_desc_lo(base + kOffKV + stage * 2 * kTileBytes + c0 * kRowBytes);
+                        const uint32_t tSh = tSh0 + c0;
+                        mma_ss_lean<0>(tSh, q_lo, k_lo, idesc);  // K = 64 as four steps of 16 (32 bytes)
+                        mma_ss_lean<1>(tSh, q_lo + 2, k_lo + 2, idesc);
+                        mma_ss_lean<1>(tSh, q_lo + 4, k_lo + 4, idesc);
+                        mma_ss_lean<1>(tSh, q_lo + 6, k_lo + 6, idesc);
+                        mma_commit(bar_s);
+                        wait_p = true;
+                        qk_c0 = c0;
+                        qk_c1 = c1;
+                        qk_stage = stage;
+                        TR_ADD(2, t_qk);
+                        TR_INC(4);
+                    }
+                    if (have_p) issue_pv();
+                }
+                if (alive && wait_p) {
+                    if ((alive = take_p())) issue_pv();
                 }
                 kv_cnt += n_tiles;
                 if (!alive) break;
@@ -605,8 +666,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 ++unit_cnt;
             }
             // nothing of this CTA may still run on the tensor pipe when TMEM is freed
-            mma_commit(bars + 8 * kBarFinal);
-            mbar_wait_bounded(bars + 8 * kBarFinal, 0, kWaitLimit);
+            mma_commit(bars + 8 * (kBarFinal + h));
+            mbar_wait_bounded(bars + 8 * (kBarFinal + h), 0, kWaitLimit);
         }
         __syncwarp();
     } else {
@@ -647,8 +708,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         };
         auto wait_free = [&](uint32_t bar, uint32_t parity) -> bool {
             if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
+            TR_T0(t_fl);
             flush();
-            return wait(bar, parity);
+            TR_ADD(1, t_fl);
+            TR_T0(t_wf);
+            const bool ok = wait(bar, parity);
+            TR_ADD(0, t_wf);
+            return ok;
         };
 
         // scheduler state (lane 0 of the first loader warp only)
@@ -724,15 +790,28 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 load_indices(idx, perm, t.k0, (t.w + 15) & ~15, t.w - 1, ltid);
                 if (!(alive = wait_free(bars + 8 * (kBarKVEmpty + stage), ((kv_cnt / kStages) & 1) ^ 1))) break;
                 const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
+                TR_T0(t_cp);
                 copy_rows(sK, Kbh, idx, ltid);
                 copy_rows(sK + kTileBytes, Vbh, idx, ltid);
+                TR_ADD(2, t_cp);
+                TR_T0(t_cs);
                 commit_and_signal(bars + 8 * (kBarKVFull + stage));
+                TR_ADD(3, t_cs);
+                TR_INC(4);
                 ++kv_cnt;
             }
         }
         flush();  // drain: signal the groups still pending
     }
 
+#ifdef MATE_TRACE
+    if (lane == 0 && (warp == 0 || warp == 4 || warp == kMmaWarp || warp == kLoadWarp0)) {  // MMA: half 0's thread
+        const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == kMmaWarp ? 2 : 3;
+        long long *o = g_trace + blockIdx.x * 32 + role * 8;
+        for (int i = 0; i < 7; ++i) o[i] = tr[i];
+        o[7] = clock64() - tr_start;
+    }
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
@@ -787,3 +866,10 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 }
 
 }  // namespace mate
+
+#ifdef MATE_TRACE
+// copies the cycle counters of the last forward launch to the host: [148 CTAs][4 roles][8]
+extern "C" int mate_debug_trace(long long *host_out) {
+    return cudaMemcpyFromSymbol(host_out, mate::g_trace, sizeof(long long) * 148 * 32) == cudaSuccess ? 0 : -4;
+}
+#endif
