@@ -395,7 +395,7 @@ int mate_attn_workspace_bytes(const mate_plan_t *plan, int d, int dtype, unsigne
     int rc = check_common(plan, d, dtype, flags, &use_tc);
     if (rc != MATE_OK) return rc;
     if (fwd_bytes) *fwd_bytes = use_tc ? mate::tc_fwd_workspace(plan, d) : 0;
-    if (bwd_bytes) *bwd_bytes = mate::simt_bwd_workspace(plan);
+    if (bwd_bytes) *bwd_bytes = use_tc ? mate::tc_bwd_workspace(plan) : mate::simt_bwd_workspace(plan);
     return MATE_OK;
 }
 
@@ -429,9 +429,11 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     const void *ptrs[] = {Q, K, V, O, LSE, dO, dQ, dK, dV};
     for (const void *p : ptrs)
         if (!aligned16(p)) return MATE_ERR_ALIGNMENT;
-    const size_t need = mate::simt_bwd_workspace(plan);
+    const size_t need = use_tc ? mate::tc_bwd_workspace(plan) : mate::simt_bwd_workspace(plan);
     if (!workspace || workspace_bytes < need) return MATE_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MATE_ERR_ALIGNMENT;
+    if (use_tc)
+        return mate::tc_bwd(plan, Q, K, V, O, LSE, dO, scale, dQ, dK, dV, workspace, (cudaStream_t)stream);
     return mate::simt_bwd(plan, Q, K, V, O, LSE, dO, d, dtype, scale, dQ, dK, dV, workspace,
                           (cudaStream_t)stream);
 }

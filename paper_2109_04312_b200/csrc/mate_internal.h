@@ -93,6 +93,10 @@ int simt_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *
 // tensor-core kernels (mate_fwd_tc.cu / mate_bwd_tc.cu)
 bool tc_supported(int d, int dtype);
 size_t tc_fwd_workspace(const mate_plan_t *plan, int d);
+size_t tc_bwd_workspace(const mate_plan_t *plan);
+int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, const void *O,
+           const float *LSE, const void *dO, float scale, void *dQ, void *dK, void *dV, void *workspace,
+           cudaStream_t stream);
 int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, float scale, void *O,
            float *LSE, void *workspace, cudaStream_t stream);
 
