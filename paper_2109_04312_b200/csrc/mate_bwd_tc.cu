@@ -143,14 +143,14 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const __nv_bfloat16 *__rest
     if (lane == 0) D[r] = acc;
 }
 
-// Rounds the fp32 sums of the split prefix rows into the outputs: one block per unit, only the
-// first part of a split unit does anything.  The rows of such a unit are prefix rows, whose view
+// Rounds the fp32 sums of the split prefix rows into the outputs: blocks (u, y) cover unit u in
+// gridDim.y slices of rows; only the first part of a split unit does anything.  The rows of such a unit are prefix rows, whose view
 // position is their original position.
 __global__ void __launch_bounds__(256) finalize_kernel(const Params p) {
     const FwdUnit un = load_unit(p.units + blockIdx.x);
     if (un.n_parts <= 1 || un.part != 0) return;
     const size_t bh = (size_t)un.b * p.H + un.h;
-    for (int i = threadIdx.x; i < un.nq * 32; i += blockDim.x) {
+    for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < un.nq * 32; i += blockDim.x * gridDim.y) {
         const int row = un.q0 + (i >> 5), c2 = i & 31;
         const float *a = p.acc32 + (bh * p.P + row) * 64 + 2 * c2;
         const size_t dst = (bh * p.N + row) * 64 + 2 * c2;
@@ -174,7 +174,7 @@ struct Cta {
 template <bool kKeySide>
 __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, int h, uint32_t &ph_s,
                              uint32_t &ph_fin) {
-    const int tid = c.tid, warp = c.warp, lane = c.lane;
+    const int tid = c.tid, warp = c.warp;
     const int r = tid & 127;         // row of the tile = lane of tensor memory
     const int hc = warp >> 2;        // which 64 columns of a column tile this thread works on
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -527,7 +527,7 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
         return MATE_ERR_CUDA;
     rowdot_kernel<<<(unsigned)((bhn + 7) / 8), 256, 0, stream>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, D, bhn);
     tc_bwd_kernel<<<plan->n_ctas, kThreads, kSmemBytes, stream>>>(p);
-    if (p.acc32) finalize_kernel<<<plan->n_fwd_units, 256, 0, stream>>>(p);
+    if (p.acc32) finalize_kernel<<<dim3(plan->n_fwd_units, 16), 256, 0, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
