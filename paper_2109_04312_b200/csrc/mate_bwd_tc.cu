@@ -12,8 +12,8 @@
 // so no gradient is accumulated across CTAs except for prefix rows whose column range was split
 // at plan time; those add fp32 partial sums into a scratch buffer that a last small kernel rounds.
 //
-// One CTA per SM, 256 threads.  Thread r (and r + 128) owns row r of a 128-row tile: lane of
-// tensor memory; warps 0-3 take columns 0-63 of a column tile, warps 4-7 columns 64-127.  Per
+// One CTA per SM, 512 threads.  Four threads (r, r + 128, r + 256, r + 384) share row r of a
+// 128-row tile, the lane of tensor memory; each takes 32 of the 128 columns of a column tile.  Per
 // column tile: two tcgen05.mma groups fill S and dP (fp32, tensor memory), the threads turn them
 // into bf16 P / dS operands written back to tensor memory, and further MMAs read those operands
 // from tensor memory and accumulate the gradients there.  Rows are gathered by view-order index
@@ -26,11 +26,15 @@
 
 namespace mate {
 
+#ifdef MATE_TRACE
+__device__ long long g_trace_bwd[148 * 16];
+#endif
+
 namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kRowBytes = 128;
 constexpr int kTileBytes = kTile * kRowBytes;  // 16 KB
 constexpr uint32_t kOffRa = 0;                 // row operand a (Q or K)
@@ -101,20 +105,20 @@ __device__ __forceinline__ FwdUnit load_unit(const FwdUnit *p) {
 }
 
 // Gathers rows of two tensors into two swizzled tiles: row rr comes from view position
-// row0 + min(rr, clamp).  32 rows per pass, 8 threads per row.
+// row0 + min(rr, clamp).  64 rows per pass, 8 threads per row.
 __device__ __forceinline__ void load_pair(uint32_t s_a, uint32_t s_b, const __nv_bfloat16 *a_bh,
                                           const __nv_bfloat16 *b_bh, const int32_t *perm, int row0,
                                           int n_rows, int clamp, int tid) {
     const int chunk = tid & 7;
-    int idx[4];
+    int idx[2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int rr = (tid >> 3) + 32 * i;
+    for (int i = 0; i < 2; ++i) {
+        const int rr = (tid >> 3) + 64 * i;
         idx[i] = rr < n_rows ? __ldg(perm + row0 + min(rr, clamp)) : -1;
     }
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int rr = (tid >> 3) + 32 * i;
+    for (int i = 0; i < 2; ++i) {
+        const int rr = (tid >> 3) + 64 * i;
         if (idx[i] >= 0) {
             const uint32_t off = rr * kRowBytes + ((chunk ^ (rr & 7)) << 4);
             cp_async16(s_a + off, a_bh + (size_t)idx[i] * 64 + chunk * 8, 16u);
@@ -169,14 +173,21 @@ struct Cta {
     uint32_t base, bars, tmem;
     int tid, warp, lane;
     volatile int *s_abort;
+#ifdef MATE_TRACE
+    long long *tr;
+#endif
 };
 
 template <bool kKeySide>
 __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, int h, uint32_t &ph_s,
                              uint32_t &ph_fin) {
     const int tid = c.tid, warp = c.warp;
+#ifdef MATE_TRACE
+    long long *tr = c.tr;
+#endif
+    TR_T0(t_item);
     const int r = tid & 127;         // row of the tile = lane of tensor memory
-    const int hc = warp >> 2;        // which 64 columns of a column tile this thread works on
+    const int cq = warp >> 2;        // which 32 columns of a column tile this thread works on
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tm = c.tmem + lane_base;
     const uint32_t bar_s = c.bars, bar_fin = c.bars + 8;
@@ -193,7 +204,7 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
     const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
 
     if (n_tiles == 0) {  // padding rows: zero gradients
-        if (row_valid && hc == 0) {
+        if (row_valid && cq == 0) {
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 if (!kKeySide) reinterpret_cast<uint4 *>(p.dQ + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
@@ -210,10 +221,20 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
     const __nv_bfloat16 *Ca_bh = (kKeySide ? p.Q : p.K) + bh * 64, *Cb_bh = (kKeySide ? p.dO : p.V) + bh * 64;
     const uint32_t sRa = c.base + kOffRa, sRb = c.base + kOffRb;
 
-    int my_lo = 0, my_hi = 0;
+    // own segment of this row and the envelope over the 32 rows of the warp
+    int my_lo = 0, my_hi = 0, w_lo_min = 0, w_lo_max = 0, w_hi_min = 0, w_hi_max = 0;
     if (nB > 0) {
         my_lo = vp.seg_lo[(size_t)un.b * p.N + t_row];
         my_hi = vp.seg_hi[(size_t)un.b * p.N + t_row];
+        w_lo_min = w_lo_max = my_lo;
+        w_hi_min = w_hi_max = my_hi;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            w_lo_min = min(w_lo_min, __shfl_xor_sync(0xffffffffu, w_lo_min, o));
+            w_lo_max = max(w_lo_max, __shfl_xor_sync(0xffffffffu, w_lo_max, o));
+            w_hi_min = min(w_hi_min, __shfl_xor_sync(0xffffffffu, w_hi_min, o));
+            w_hi_max = max(w_hi_max, __shfl_xor_sync(0xffffffffu, w_hi_max, o));
+        }
     }
     float row_lse2 = 0.f, row_D = 0.f;  // query side: this row's LSE (log2 domain) and D
     if (!kKeySide) {
@@ -267,10 +288,14 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
     while (i < n_tiles) {
         const int st = n_done & 1;
         const uint32_t sCa = c.base + kOffC + st * 2 * kTileBytes, sCb = sCa + kTileBytes;
+        TR_T0(t_ld);
         cp_async_wait_all();
         fence_proxy_async();
         tc_fence_before();
         __syncthreads();  // the tile has landed; everybody is done with tensor memory of the previous tile
+        TR_ADD(0, t_ld);
+        TR_INC(7);
+        TR_T0(t_m1);
 
         if (tid == 0) {
             tc_fence_after();
@@ -287,6 +312,8 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
             mma_ss_lean<1>(c.tmem + kTmT + c0, rb + 6, cb + 6, idesc);
             mma_commit(bar_s);  // also covers the gradient MMAs of the previous tile
         }
+        TR_ADD(1, t_m1);
+        TR_T0(t_ws);
         const bool ok = wait(bar_s, ph_s);
         ph_s ^= 1;
         if (__syncthreads_or(!ok)) {
@@ -294,6 +321,8 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
             break;
         }
         tc_fence_after();
+        TR_ADD(2, t_ws);
+        TR_T0(t_pf);
 
         // the other stage is free now (its readers completed with the commit above): next tile
         TileInfo tn;
@@ -302,41 +331,64 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
         if (i_next < n_tiles) load_cols(tn, st ^ 1);
         cp_async_commit();
 
-        // this thread's columns [r_lo, r_hi) of the tile
-        int r_lo, r_hi;
+        TR_ADD(3, t_pf);
+        TR_T0(t_cmp);
+        // this thread's columns [r_lo, r_hi) of the tile and the warp's envelope
+        int r_lo, r_hi, e_lo_min, e_lo_max, e_hi_min, e_hi_max;
         if (!t.is_b) {
-            r_lo = 0;
-            r_hi = un.kA_end - t.k0;
+            r_lo = e_lo_min = e_lo_max = 0;
+            r_hi = e_hi_min = e_hi_max = un.kA_end - t.k0;
         } else {
             r_lo = my_lo - t.k0;
             r_hi = my_hi - t.k0;
+            e_lo_min = w_lo_min - t.k0;
+            e_lo_max = w_lo_max - t.k0;
+            e_hi_min = w_hi_min - t.k0;
+            e_hi_max = w_hi_max - t.k0;
         }
         const uint32_t r_span = (uint32_t)max(r_hi - r_lo, 0);
-        const float *vec = reinterpret_cast<const float *>(__cvta_shared_to_generic(c.base + kOffVec + st * 1024));
+        const float4 *vec4 = reinterpret_cast<const float4 *>(__cvta_shared_to_generic(c.base + kOffVec + st * 1024));
 
-#pragma unroll 1
-        for (int cc = 0; cc < 2; ++cc) {
-            const int cb = hc * 64 + cc * 32;
-            if (cb >= c1 || cb + 32 <= c0) continue;  // outside the columns the MMAs touch
-            uint32_t sv[32], tv[32];
-            tmem_ld32(tm + kTmS + cb, sv);
-            tmem_ld32(tm + kTmT + cb, tv);
-            tc_wait_ld();
+        const int cb = cq * 32;  // this thread's 32 columns
+        if (cb < c1 && cb + 32 > c0) {  // inside the columns the MMAs touch
             uint32_t pk_p[16], pk_ds[16];
+            if (cb + 32 <= e_lo_min || cb >= e_hi_max) {
+                // no row of the warp has a pair here
 #pragma unroll
-            for (int e = 0; e < 32; e += 2) {
-                float pv[2], dsv[2];
+                for (int e = 0; e < 16; ++e) pk_p[e] = pk_ds[e] = 0u;
+            } else {
+                uint32_t sv[32], tv[32];
+                tmem_ld32(tm + kTmS + cb, sv);
+                tmem_ld32(tm + kTmT + cb, tv);
+                tc_wait_ld();
+                const bool full = cb >= e_lo_max && cb + 32 <= e_hi_min;
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    const float lse2 = kKeySide ? vec[cb + e + q] : row_lse2;
-                    const float Dv = kKeySide ? vec[128 + cb + e + q] : row_D;
-                    const bool on = (uint32_t)(cb + e + q - r_lo) < r_span;
-                    const float x = fmaf(__uint_as_float(sv[e + q]), p.scale_log2, -lse2);
-                    pv[q] = on ? ex2(x) : 0.f;
-                    dsv[q] = pv[q] * (__uint_as_float(tv[e + q]) - Dv);
+                for (int e = 0; e < 32; e += 4) {
+                    float lse2[4], Dv[4];
+                    if (kKeySide) {
+                        const float4 a = vec4[(cb + e) >> 2], d4 = vec4[32 + ((cb + e) >> 2)];
+                        lse2[0] = a.x; lse2[1] = a.y; lse2[2] = a.z; lse2[3] = a.w;
+                        Dv[0] = d4.x; Dv[1] = d4.y; Dv[2] = d4.z; Dv[3] = d4.w;
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            lse2[q] = row_lse2;
+                            Dv[q] = row_D;
+                        }
+                    }
+                    float pv[4], dsv[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float x = fmaf(__uint_as_float(sv[e + q]), p.scale_log2, -lse2[q]);
+                        pv[q] = ex2(x);
+                        if (!full && (uint32_t)(cb + e + q - r_lo) >= r_span) pv[q] = 0.f;
+                        dsv[q] = pv[q] * (__uint_as_float(tv[e + q]) - Dv[q]);
+                    }
+                    pk_p[e >> 1] = pack_bf16(pv[0], pv[1]);
+                    pk_p[(e >> 1) + 1] = pack_bf16(pv[2], pv[3]);
+                    pk_ds[e >> 1] = pack_bf16(dsv[0], dsv[1]);
+                    pk_ds[(e >> 1) + 1] = pack_bf16(dsv[2], dsv[3]);
                 }
-                pk_p[e >> 1] = pack_bf16(pv[0], pv[1]);
-                pk_ds[e >> 1] = pack_bf16(dsv[0], dsv[1]);
             }
             if (kKeySide) {
                 tmem_st16(tm + kTmA1 + (cb >> 1), pk_p);
@@ -348,6 +400,8 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
         tc_wait_st();
         tc_fence_before();
         __syncthreads();
+        TR_ADD(4, t_cmp);
+        TR_T0(t_m2);
 
         if (tid == 0) {
             tc_fence_after();
@@ -365,6 +419,7 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
                 }
             }
         }
+        TR_ADD(5, t_m2);
         ++n_done;
         i = i_next;
         t = tn;
@@ -380,22 +435,22 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
     ph_fin ^= 1;
     if (__syncthreads_or(!ok)) return;
     tc_fence_after();
-    if (kKeySide || hc == 0) {
-        // warps 0-3: accumulator 1 (dQ or dV); warps 4-7 (key side): accumulator 2 (dK)
-        const uint32_t tacc = tm + (hc == 0 ? kTmAcc1 : kTmAcc2);
-        const float mul = (!kKeySide || hc == 1) ? p.scale : 1.f;
-        __nv_bfloat16 *out = !kKeySide ? p.dQ : (hc == 0 ? p.dV : p.dK);
-        const int plane = !kKeySide ? 0 : (hc == 0 ? 2 : 1);
-        uint32_t a0[32], a1[32];
+    if (kKeySide || cq < 2) {
+        // column quarters 0, 1: the two halves of accumulator 1 (dQ or dV); 2, 3 (key side): of accumulator 2 (dK)
+        const int half = cq & 1;
+        const uint32_t tacc = tm + (cq < 2 ? kTmAcc1 : kTmAcc2) + 32 * half;
+        const float mul = (!kKeySide || cq >= 2) ? p.scale : 1.f;
+        __nv_bfloat16 *out = !kKeySide ? p.dQ : (cq < 2 ? p.dV : p.dK);
+        const int plane = !kKeySide ? 0 : (cq < 2 ? 2 : 1);
+        uint32_t a0[32];
         tmem_ld32(tacc, a0);
-        tmem_ld32(tacc + 32, a1);
         tc_wait_ld();
         if (row_valid) {
             if (un.n_parts == 1) {
-                uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64);
+                uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + 32 * half);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const uint32_t *src = q < 4 ? a0 + 8 * q : a1 + 8 * (q - 4);
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t *src = a0 + 8 * q;
                     dst[q] = make_uint4(pack_bf16(__uint_as_float(src[0]) * mul, __uint_as_float(src[1]) * mul),
                                         pack_bf16(__uint_as_float(src[2]) * mul, __uint_as_float(src[3]) * mul),
                                         pack_bf16(__uint_as_float(src[4]) * mul, __uint_as_float(src[5]) * mul),
@@ -403,16 +458,15 @@ __device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, i
                 }
             } else {
                 // split prefix rows: view position = original position < P
-                float *dst = p.acc32 + plane * p.plane + (((size_t)un.b * p.H + un.h) * p.P + orig) * 64;
+                float *dst = p.acc32 + plane * p.plane + (((size_t)un.b * p.H + un.h) * p.P + orig) * 64 + 32 * half;
 #pragma unroll
                 for (int e = 0; e < 32; ++e) atomicAdd(dst + e, __uint_as_float(a0[e]) * mul);
-#pragma unroll
-                for (int e = 0; e < 32; ++e) atomicAdd(dst + 32 + e, __uint_as_float(a1[e]) * mul);
             }
         }
     }
     tc_fence_before();
     __syncthreads();  // tensor memory and the row operand tiles are free for the next item
+    TR_ADD(6, t_item);
 }
 
 // Work items: (unit, half, side), taken from a counter in the order of the plan's unit list
@@ -446,6 +500,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
     tc_fence_after();
     c.tmem = *tmem_slot;
 
+#ifdef MATE_TRACE
+    long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    c.tr = tr;
+    const long long tr_start = clock64();
+#endif
     uint32_t ph_s = 0, ph_fin = 0;
     const int n_items = p.n_units * 4;
     while (true) {
@@ -460,6 +519,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
         else process_item<false>(p, c, un, h, ph_s, ph_fin);
     }
 
+#ifdef MATE_TRACE
+    if (c.tid == 0 || c.tid == 255) {
+        long long *o = g_trace_bwd + blockIdx.x * 16 + (c.tid == 0 ? 0 : 8);
+        for (int i = 0; i < 8; ++i) o[i] = tr[i];
+        if (c.tid == 0) o[6] = clock64() - tr_start;  // thread 0: total instead of the item sum
+    }
+#endif
     // nothing of this CTA may still run on the tensor pipe when tensor memory is freed
     if (*c.s_abort && c.tid == 0) {
         mma_commit(c.bars + 8);
@@ -532,3 +598,10 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 }
 
 }  // namespace mate
+
+#ifdef MATE_TRACE
+// copies the cycle counters of the last backward launch to the host: [148 CTAs][2 threads][8]
+extern "C" int mate_debug_trace_bwd(long long *host_out) {
+    return cudaMemcpyFromSymbol(host_out, mate::g_trace_bwd, sizeof(long long) * 148 * 16) == cudaSuccess ? 0 : -4;
+}
+#endif

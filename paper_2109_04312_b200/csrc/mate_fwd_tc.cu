@@ -25,17 +25,8 @@
 
 namespace mate {
 
-// Optional cycle counters (compile with -DMATE_TRACE): per CTA and role, clock64() time spent in
-// the marked regions.  Profiling aid only; compiled out of the library.
 #ifdef MATE_TRACE
 __device__ long long g_trace[148 * 32];
-#define TR_T0(var) const long long var = clock64()
-#define TR_ADD(cat, var) tr[cat] += clock64() - (var)
-#define TR_INC(cat) tr[cat] += 1
-#else
-#define TR_T0(var)
-#define TR_ADD(cat, var)
-#define TR_INC(cat)
 #endif
 
 namespace {

@@ -101,3 +101,16 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
            float *LSE, void *workspace, cudaStream_t stream);
 
 }  // namespace mate
+
+// Optional cycle counters (compile with -DMATE_TRACE): clock64() time spent in marked regions of
+// the tensor-core kernels, per CTA and role, in a local array `tr`.  Profiling aid only; compiled
+// out of the library.
+#ifdef MATE_TRACE
+#define TR_T0(var) const long long var = clock64()
+#define TR_ADD(cat, var) tr[cat] += clock64() - (var)
+#define TR_INC(cat) tr[cat] += 1
+#else
+#define TR_T0(var)
+#define TR_ADD(cat, var)
+#define TR_INC(cat)
+#endif
