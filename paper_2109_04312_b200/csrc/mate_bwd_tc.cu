@@ -12,14 +12,21 @@
 // so no gradient is accumulated across CTAs except for prefix rows whose column range was split
 // at plan time; those add fp32 partial sums into a scratch buffer that a last small kernel rounds.
 //
-// One CTA per SM, 512 threads.  Four threads (r, r + 128, r + 256, r + 384) share row r of a
-// 128-row tile, the lane of tensor memory; each takes 32 of the 128 columns of a column tile.  Per
-// column tile: two tcgen05.mma groups fill S and dP (fp32, tensor memory), the threads turn them
-// into bf16 P / dS operands written back to tensor memory, and further MMAs read those operands
-// from tensor memory and accumulate the gradients there.  Rows are gathered by view-order index
-// with 16-byte cp.async into 128-byte swizzled shared memory (next tile in flight during the
-// arithmetic) and scattered back in the epilogue.
+// One persistent, warp-specialised CTA per SM (20 warps); work items (unit, half, side) are handed
+// out through a counter in the order of the plan's unit list.
+//   warps 0-15  arithmetic: four threads (r, r + 128, r + 256, r + 384) share row r of the 128-row
+//               tile, the lane of tensor memory; each takes 32 of the 128 columns of a column tile.
+//               S and dP (fp32) come out of tensor memory, P / dS (bf16 pairs) go back into it as
+//               MMA operands.
+//   warp  16    one thread issues every tcgen05.mma: S and dP of tile n + 1 go ahead of the
+//               gradient MMAs of tile n, which then run under the arithmetic of tile n + 1
+//   warps 17-19 loaders: gather rows by view-order index with 16-byte cp.async into 128-byte
+//               swizzled shared memory (row operands double buffered, column tiles in a ring of 3)
+// The gradients accumulate in tensor memory and are scattered to the rows' original positions in
+// the epilogue.
 #include <cuda_bf16.h>
+
+#include <type_traits>
 
 #include "mate_internal.h"
 #include "sm100_ptx.cuh"
@@ -27,22 +34,44 @@
 namespace mate {
 
 #ifdef MATE_TRACE
-__device__ long long g_trace_bwd[148 * 16];
+__device__ long long g_trace_bwd[148 * 32];
 #endif
 
 namespace {
 
 using namespace ptx;
 
-constexpr int kThreads = 512;
+constexpr int kComputeWarps = 16;
+constexpr int kMmaWarp = 16;
+constexpr int kLoadWarp0 = 17;
+constexpr int kLoadWarps = 3;
+constexpr int kLoadThreads = 32 * kLoadWarps;
+constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
+constexpr int kStages = 3;  // ring of column tiles
+constexpr int kLag = 2;     // loader: copy groups in flight behind the newest one
 constexpr int kRowBytes = 128;
 constexpr int kTileBytes = kTile * kRowBytes;  // 16 KB
-constexpr uint32_t kOffRa = 0;                 // row operand a (Q or K)
-constexpr uint32_t kOffRb = kTileBytes;        // row operand b (dO or V)
-constexpr uint32_t kOffC = 2 * kTileBytes;     // [2 stages] x (Ca 16 KB, Cb 16 KB)
-constexpr uint32_t kOffVec = kOffC + 4 * kTileBytes;  // [2 stages] x (128 lse, 128 D) floats
-constexpr uint32_t kOffBar = kOffVec + 2 * 2 * 128 * 4;
-constexpr uint32_t kSmemBytes = kOffBar + 128 + 1024;
+constexpr uint32_t kOffR = 0;                  // [2 buffers] x (Ra: Q or K, Rb: dO or V), 16 KB each
+constexpr uint32_t kOffC = 4 * kTileBytes;     // [kStages] x (Ca 16 KB, Cb 16 KB)
+constexpr uint32_t kOffVec = kOffC + kStages * 2 * kTileBytes;  // [kStages] x (128 lse, 128 D) floats
+constexpr uint32_t kOffBar = kOffVec + kStages * 1024;
+constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;
+// barrier slots (8 bytes each) behind kOffBar
+enum {
+    kBarRFull = 0,    // [2] loaders -> MMA                  (count: loader warps)
+    kBarREmpty = 2,   // [2] MMA commit -> loaders           (count 1)
+    kBarCFull = 4,    // [kStages] loaders -> MMA            (count: loader warps)
+    kBarCEmpty = 7,   // [kStages] MMA commit -> loaders     (count 1)
+    kBarSFull = 10,   // MMA commit -> arithmetic: S and dP of a tile are complete (count 1)
+    kBarAFull = 11,   // arithmetic -> MMA: the bf16 operands of a tile are written (count: one per warp)
+    kBarGDone = 12,   // MMA commit -> arithmetic: the gradient MMAs of a tile are complete (count 1)
+    kBarFinal = 13,
+    kBarSchedFull = 14,   // [kSchedDepth] scheduler -> every warp (count 1)
+    kBarSchedEmpty = 18,  // [kSchedDepth] every warp -> scheduler (count kSchedReaders)
+    kNumBars = 22
+};
+constexpr int kSchedDepth = 4;
+constexpr int kSchedReaders = kComputeWarps + 1 + kLoadWarps;
 // tensor memory columns
 constexpr uint32_t kTmS = 0, kTmT = 128, kTmA1 = 256, kTmA2 = 320, kTmAcc1 = 384, kTmAcc2 = 448;
 constexpr uint32_t kWaitLimit = 4096;  // tries (up to 1 ms each) before a wait gives up
@@ -85,14 +114,14 @@ __device__ __forceinline__ TileInfo tile_info(const FwdUnit &u, int i, int nA) {
     }
     return t;
 }
-// Columns [c0, c1) of the tile (multiples of 16) that half h of the unit needs.
-__device__ __forceinline__ void half_cols(const FwdUnit &u, int h, const TileInfo &t, int &c0, int &c1) {
+// Columns [c0, c1) of the tile (multiples of 16) needed by a half whose rows' segments span keys [lo, hi).
+__device__ __forceinline__ void half_cols(int lo, int hi, const TileInfo &t, int &c0, int &c1) {
     if (!t.is_b) {
         c0 = 0;
         c1 = (t.w + 15) & ~15;
     } else {
-        c0 = (max(u.lo[h], t.k0) - t.k0) & ~15;
-        c1 = (min(u.hi[h], t.k0 + t.w) - t.k0 + 15) & ~15;
+        c0 = (max(lo, t.k0) - t.k0) & ~15;
+        c1 = (min(hi, t.k0 + t.w) - t.k0 + 15) & ~15;
     }
 }
 __device__ __forceinline__ FwdUnit load_unit(const FwdUnit *p) {
@@ -104,21 +133,26 @@ __device__ __forceinline__ FwdUnit load_unit(const FwdUnit *p) {
     return u;
 }
 
-// Gathers rows of two tensors into two swizzled tiles: row rr comes from view position
-// row0 + min(rr, clamp).  64 rows per pass, 8 threads per row.
-__device__ __forceinline__ void load_pair(uint32_t s_a, uint32_t s_b, const __nv_bfloat16 *a_bh,
-                                          const __nv_bfloat16 *b_bh, const int32_t *perm, int row0,
-                                          int n_rows, int clamp, int tid) {
-    const int chunk = tid & 7;
-    int idx[2];
+// The loaders copy a tile of up to 128 rows (128 B each) of two tensors in passes of kRowsPerPass
+// rows, 8 threads per row.  Row rr of the tile comes from view position row0 + min(rr, clamp); its
+// original position is looked up first for every pass, then the 16-byte copies follow.
+constexpr int kRowsPerPass = kLoadThreads / 8;
+constexpr int kPasses = (kTile + kRowsPerPass - 1) / kRowsPerPass;
+
+__device__ __forceinline__ void load_indices(int (&idx)[kPasses], const int32_t *perm, int row0,
+                                             int n_rows, int clamp, int ltid) {
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int rr = (tid >> 3) + 64 * i;
+    for (int i = 0; i < kPasses; ++i) {
+        const int rr = (ltid >> 3) + kRowsPerPass * i;
         idx[i] = rr < n_rows ? __ldg(perm + row0 + min(rr, clamp)) : -1;
     }
+}
+__device__ __forceinline__ void copy_pair(uint32_t s_a, uint32_t s_b, const __nv_bfloat16 *a_bh,
+                                          const __nv_bfloat16 *b_bh, const int (&idx)[kPasses], int ltid) {
+    const int chunk = ltid & 7;
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int rr = (tid >> 3) + 64 * i;
+    for (int i = 0; i < kPasses; ++i) {
+        const int rr = (ltid >> 3) + kRowsPerPass * i;
         if (idx[i] >= 0) {
             const uint32_t off = rr * kRowBytes + ((chunk ^ (rr & 7)) << 4);
             cp_async16(s_a + off, a_bh + (size_t)idx[i] * 64 + chunk * 8, 16u);
@@ -167,373 +201,573 @@ __global__ void __launch_bounds__(256) finalize_kernel(const Params p) {
     }
 }
 
-// One work item: half `h` (128 rows) of unit `un`, on the query side (kKeySide = false: rows are
-// queries, dQ is produced) or on the key side (rows are keys, dK and dV are produced).
-struct Cta {
-    uint32_t base, bars, tmem;
-    int tid, warp, lane;
-    volatile int *s_abort;
-#ifdef MATE_TRACE
-    long long *tr;
-#endif
+// Everything an item needs that does not depend on the role of the warp.
+struct Item {
+    FwdUnit un;
+    int h, n_tiles, nA, rows_h, row0, lo, hi;  // lo, hi: un.lo[h], un.hi[h]
+    bool key_side;
 };
-
-template <bool kKeySide>
-__device__ void process_item(const Params &p, const Cta &c, const FwdUnit &un, int h, uint32_t &ph_s,
-                             uint32_t &ph_fin) {
-    const int tid = c.tid, warp = c.warp;
-#ifdef MATE_TRACE
-    long long *tr = c.tr;
-#endif
-    TR_T0(t_item);
-    const int r = tid & 127;         // row of the tile = lane of tensor memory
-    const int cq = warp >> 2;        // which 32 columns of a column tile this thread works on
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t tm = c.tmem + lane_base;
-    const uint32_t bar_s = c.bars, bar_fin = c.bars + 8;
-
-    const int rows_h = max(0, min(kTile, un.nq - h * kTile));
-    if (rows_h == 0) return;
-    const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
-    const int32_t *perm = vp.perm + (size_t)un.b * p.N;
-    const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
-    const bool row_valid = r < rows_h;
-    const int row0 = un.q0 + h * kTile;
-    const int t_row = row0 + min(r, rows_h - 1);  // rows past the end shadow the last one
-    const int orig = perm[t_row];
-    const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
-
-    if (n_tiles == 0) {  // padding rows: zero gradients
-        if (row_valid && cq == 0) {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                if (!kKeySide) reinterpret_cast<uint4 *>(p.dQ + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
-                if (kKeySide) {
-                    reinterpret_cast<uint4 *>(p.dK + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
-                    reinterpret_cast<uint4 *>(p.dV + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
-                }
-            }
-        }
-        return;
+__device__ __forceinline__ Item make_item(const Params &p, int it) {
+    Item x;
+    x.un = load_unit(p.units + (it >> 2));
+    x.h = it & 1;
+    x.key_side = (it & 2) != 0;
+    x.nA = n_tiles_a(x.un);
+    x.n_tiles = x.nA + n_tiles_b(x.un);
+    x.rows_h = max(0, min(kTile, x.un.nq - x.h * kTile));
+    x.row0 = x.un.q0 + x.h * kTile;
+    x.lo = x.h ? x.un.lo[1] : x.un.lo[0];
+    x.hi = x.h ? x.un.hi[1] : x.un.hi[0];
+    return x;
+}
+// Next tile at or after i that this half takes part in (n_tiles if none).
+__device__ __forceinline__ int next_tile(const Item &x, int i, TileInfo &t, int &c0, int &c1) {
+    for (; i < x.n_tiles; ++i) {
+        t = tile_info(x.un, i, x.nA);
+        half_cols(x.lo, x.hi, t, c0, c1);
+        if (c1 > c0) return i;
     }
-
-    const __nv_bfloat16 *Ra_bh = (kKeySide ? p.K : p.Q) + bh * 64, *Rb_bh = (kKeySide ? p.V : p.dO) + bh * 64;
-    const __nv_bfloat16 *Ca_bh = (kKeySide ? p.Q : p.K) + bh * 64, *Cb_bh = (kKeySide ? p.dO : p.V) + bh * 64;
-    const uint32_t sRa = c.base + kOffRa, sRb = c.base + kOffRb;
-
-    // own segment of this row and the envelope over the 32 rows of the warp
-    int my_lo = 0, my_hi = 0, w_lo_min = 0, w_lo_max = 0, w_hi_min = 0, w_hi_max = 0;
-    if (nB > 0) {
-        my_lo = vp.seg_lo[(size_t)un.b * p.N + t_row];
-        my_hi = vp.seg_hi[(size_t)un.b * p.N + t_row];
-        w_lo_min = w_lo_max = my_lo;
-        w_hi_min = w_hi_max = my_hi;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            w_lo_min = min(w_lo_min, __shfl_xor_sync(0xffffffffu, w_lo_min, o));
-            w_lo_max = max(w_lo_max, __shfl_xor_sync(0xffffffffu, w_lo_max, o));
-            w_hi_min = min(w_hi_min, __shfl_xor_sync(0xffffffffu, w_hi_min, o));
-            w_hi_max = max(w_hi_max, __shfl_xor_sync(0xffffffffu, w_hi_max, o));
-        }
-    }
-    float row_lse2 = 0.f, row_D = 0.f;  // query side: this row's LSE (log2 domain) and D
-    if (!kKeySide) {
-        row_lse2 = p.LSE[bh + orig] * 1.4426950408889634f;
-        row_D = p.D[bh + orig];
-    }
-
-    // participating tiles of this half, in order
-    auto next_tile = [&](int i, TileInfo &t, int &c0, int &c1) -> int {
-        for (; i < n_tiles; ++i) {
-            t = tile_info(un, i, nA);
-            half_cols(un, h, t, c0, c1);
-            if (c1 > c0) return i;
-        }
-        return n_tiles;
-    };
-    // column tile `t` into stage `st`: rows [0, n16) of both operands, and on the key side the
-    // LSE / D of the query columns
-    auto load_cols = [&](const TileInfo &t, int st) {
-        const int n16 = (t.w + 15) & ~15;
-        const uint32_t sCa = c.base + kOffC + st * 2 * kTileBytes;
-        load_pair(sCa, sCa + kTileBytes, Ca_bh, Cb_bh, perm, t.k0, n16, t.w - 1, tid);
-        if (kKeySide && tid < kTile) {
-            float *vec = reinterpret_cast<float *>(__cvta_shared_to_generic(c.base + kOffVec + st * 1024));
-            const int o = perm[t.k0 + min(tid, t.w - 1)];
-            vec[tid] = p.LSE[bh + o] * 1.4426950408889634f;
-            vec[128 + tid] = p.D[bh + o];
-        }
-    };
-
-    bool failed = false;
-    auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
-        for (uint32_t it = 0; it < kWaitLimit; ++it) {
-            if (mbar_try_wait(bar, parity)) return true;
-            if (*c.s_abort) return false;
-        }
-        *c.s_abort = 1;
-        atomicOr(p.status + 1, 1);
-        return false;
-    };
-
-    TileInfo t;
-    int c0 = 0, c1 = 0;
-    int i = next_tile(0, t, c0, c1);
-    // prologue: row operands and the first column tile
-    load_pair(sRa, sRb, Ra_bh, Rb_bh, perm, row0, kTile, rows_h - 1, tid);
-    if (i < n_tiles) load_cols(t, 0);
-    cp_async_commit();
-
-    int n_done = 0;
-    while (i < n_tiles) {
-        const int st = n_done & 1;
-        const uint32_t sCa = c.base + kOffC + st * 2 * kTileBytes, sCb = sCa + kTileBytes;
-        TR_T0(t_ld);
-        cp_async_wait_all();
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();  // the tile has landed; everybody is done with tensor memory of the previous tile
-        TR_ADD(0, t_ld);
-        TR_INC(7);
-        TR_T0(t_m1);
-
-        if (tid == 0) {
-            tc_fence_after();
-            const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
-            const uint32_t ra = smem_desc_lo(sRa), rb = smem_desc_lo(sRb);
-            const uint32_t ca = smem_desc_lo(sCa + c0 * kRowBytes), cb = smem_desc_lo(sCb + c0 * kRowBytes);
-            mma_ss_lean<0>(c.tmem + kTmS + c0, ra, ca, idesc);  // S = Ra Ca^T, K = 64 as four steps of 16
-            mma_ss_lean<1>(c.tmem + kTmS + c0, ra + 2, ca + 2, idesc);
-            mma_ss_lean<1>(c.tmem + kTmS + c0, ra + 4, ca + 4, idesc);
-            mma_ss_lean<1>(c.tmem + kTmS + c0, ra + 6, ca + 6, idesc);
-            mma_ss_lean<0>(c.tmem + kTmT + c0, rb, cb, idesc);  // dP = Rb Cb^T
-            mma_ss_lean<1>(c.tmem + kTmT + c0, rb + 2, cb + 2, idesc);
-            mma_ss_lean<1>(c.tmem + kTmT + c0, rb + 4, cb + 4, idesc);
-            mma_ss_lean<1>(c.tmem + kTmT + c0, rb + 6, cb + 6, idesc);
-            mma_commit(bar_s);  // also covers the gradient MMAs of the previous tile
-        }
-        TR_ADD(1, t_m1);
-        TR_T0(t_ws);
-        const bool ok = wait(bar_s, ph_s);
-        ph_s ^= 1;
-        if (__syncthreads_or(!ok)) {
-            failed = true;
-            break;
-        }
-        tc_fence_after();
-        TR_ADD(2, t_ws);
-        TR_T0(t_pf);
-
-        // the other stage is free now (its readers completed with the commit above): next tile
-        TileInfo tn;
-        int n0 = 0, n1 = 0;
-        const int i_next = next_tile(i + 1, tn, n0, n1);
-        if (i_next < n_tiles) load_cols(tn, st ^ 1);
-        cp_async_commit();
-
-        TR_ADD(3, t_pf);
-        TR_T0(t_cmp);
-        // this thread's columns [r_lo, r_hi) of the tile and the warp's envelope
-        int r_lo, r_hi, e_lo_min, e_lo_max, e_hi_min, e_hi_max;
-        if (!t.is_b) {
-            r_lo = e_lo_min = e_lo_max = 0;
-            r_hi = e_hi_min = e_hi_max = un.kA_end - t.k0;
-        } else {
-            r_lo = my_lo - t.k0;
-            r_hi = my_hi - t.k0;
-            e_lo_min = w_lo_min - t.k0;
-            e_lo_max = w_lo_max - t.k0;
-            e_hi_min = w_hi_min - t.k0;
-            e_hi_max = w_hi_max - t.k0;
-        }
-        const uint32_t r_span = (uint32_t)max(r_hi - r_lo, 0);
-        const float4 *vec4 = reinterpret_cast<const float4 *>(__cvta_shared_to_generic(c.base + kOffVec + st * 1024));
-
-        const int cb = cq * 32;  // this thread's 32 columns
-        if (cb < c1 && cb + 32 > c0) {  // inside the columns the MMAs touch
-            uint32_t pk_p[16], pk_ds[16];
-            if (cb + 32 <= e_lo_min || cb >= e_hi_max) {
-                // no row of the warp has a pair here
-#pragma unroll
-                for (int e = 0; e < 16; ++e) pk_p[e] = pk_ds[e] = 0u;
-            } else {
-                uint32_t sv[32], tv[32];
-                tmem_ld32(tm + kTmS + cb, sv);
-                tmem_ld32(tm + kTmT + cb, tv);
-                tc_wait_ld();
-                const bool full = cb >= e_lo_max && cb + 32 <= e_hi_min;
-#pragma unroll
-                for (int e = 0; e < 32; e += 4) {
-                    float lse2[4], Dv[4];
-                    if (kKeySide) {
-                        const float4 a = vec4[(cb + e) >> 2], d4 = vec4[32 + ((cb + e) >> 2)];
-                        lse2[0] = a.x; lse2[1] = a.y; lse2[2] = a.z; lse2[3] = a.w;
-                        Dv[0] = d4.x; Dv[1] = d4.y; Dv[2] = d4.z; Dv[3] = d4.w;
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            lse2[q] = row_lse2;
-                            Dv[q] = row_D;
-                        }
-                    }
-                    float pv[4], dsv[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float x = fmaf(__uint_as_float(sv[e + q]), p.scale_log2, -lse2[q]);
-                        pv[q] = ex2(x);
-                        if (!full && (uint32_t)(cb + e + q - r_lo) >= r_span) pv[q] = 0.f;
-                        dsv[q] = pv[q] * (__uint_as_float(tv[e + q]) - Dv[q]);
-                    }
-                    pk_p[e >> 1] = pack_bf16(pv[0], pv[1]);
-                    pk_p[(e >> 1) + 1] = pack_bf16(pv[2], pv[3]);
-                    pk_ds[e >> 1] = pack_bf16(dsv[0], dsv[1]);
-                    pk_ds[(e >> 1) + 1] = pack_bf16(dsv[2], dsv[3]);
-                }
-            }
-            if (kKeySide) {
-                tmem_st16(tm + kTmA1 + (cb >> 1), pk_p);
-                tmem_st16(tm + kTmA2 + (cb >> 1), pk_ds);
-            } else {
-                tmem_st16(tm + kTmA1 + (cb >> 1), pk_ds);
-            }
-        }
-        tc_wait_st();
-        tc_fence_before();
-        __syncthreads();
-        TR_ADD(4, t_cmp);
-        TR_T0(t_m2);
-
-        if (tid == 0) {
-            tc_fence_after();
-            const uint32_t idesc = idesc_bf16(128, 64, 0, 1);  // B = 16 rows of the column tile x 64, MN-major
-            const int ks0 = c0 >> 4, ks1 = c1 >> 4;
-            for (int ks = ks0; ks < ks1; ++ks) {
-                const uint32_t acc = (n_done > 0 || ks > ks0) ? 1u : 0u;
-                if (kKeySide) {
-                    // dV += P^T dO, dK += dS^T Q
-                    mma_ts_lean_flag(c.tmem + kTmAcc1, c.tmem + kTmA1 + ks * 8, smem_desc_lo(sCb + ks * 16 * kRowBytes), idesc, acc);
-                    mma_ts_lean_flag(c.tmem + kTmAcc2, c.tmem + kTmA2 + ks * 8, smem_desc_lo(sCa + ks * 16 * kRowBytes), idesc, acc);
-                } else {
-                    // dQ += dS K
-                    mma_ts_lean_flag(c.tmem + kTmAcc1, c.tmem + kTmA1 + ks * 8, smem_desc_lo(sCa + ks * 16 * kRowBytes), idesc, acc);
-                }
-            }
-        }
-        TR_ADD(5, t_m2);
-        ++n_done;
-        i = i_next;
-        t = tn;
-        c0 = n0;
-        c1 = n1;
-    }
-    cp_async_wait_all();
-    if (failed) return;
-
-    // epilogue: wait for the last gradient MMAs, then scatter the rows (or add split partial sums)
-    if (tid == 0) mma_commit(bar_fin);
-    const bool ok = wait(bar_fin, ph_fin);
-    ph_fin ^= 1;
-    if (__syncthreads_or(!ok)) return;
-    tc_fence_after();
-    if (kKeySide || cq < 2) {
-        // column quarters 0, 1: the two halves of accumulator 1 (dQ or dV); 2, 3 (key side): of accumulator 2 (dK)
-        const int half = cq & 1;
-        const uint32_t tacc = tm + (cq < 2 ? kTmAcc1 : kTmAcc2) + 32 * half;
-        const float mul = (!kKeySide || cq >= 2) ? p.scale : 1.f;
-        __nv_bfloat16 *out = !kKeySide ? p.dQ : (cq < 2 ? p.dV : p.dK);
-        const int plane = !kKeySide ? 0 : (cq < 2 ? 2 : 1);
-        uint32_t a0[32];
-        tmem_ld32(tacc, a0);
-        tc_wait_ld();
-        if (row_valid) {
-            if (un.n_parts == 1) {
-                uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + 32 * half);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t *src = a0 + 8 * q;
-                    dst[q] = make_uint4(pack_bf16(__uint_as_float(src[0]) * mul, __uint_as_float(src[1]) * mul),
-                                        pack_bf16(__uint_as_float(src[2]) * mul, __uint_as_float(src[3]) * mul),
-                                        pack_bf16(__uint_as_float(src[4]) * mul, __uint_as_float(src[5]) * mul),
-                                        pack_bf16(__uint_as_float(src[6]) * mul, __uint_as_float(src[7]) * mul));
-                }
-            } else {
-                // split prefix rows: view position = original position < P
-                float *dst = p.acc32 + plane * p.plane + (((size_t)un.b * p.H + un.h) * p.P + orig) * 64 + 32 * half;
-#pragma unroll
-                for (int e = 0; e < 32; ++e) atomicAdd(dst + e, __uint_as_float(a0[e]) * mul);
-            }
-        }
-    }
-    tc_fence_before();
-    __syncthreads();  // tensor memory and the row operand tiles are free for the next item
-    TR_ADD(6, t_item);
+    return x.n_tiles;
 }
 
-// Work items: (unit, half, side), taken from a counter in the order of the plan's unit list
-// (largest units first).
 __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
-    Cta c;
-    c.base = (raw + 1023u) & ~1023u;
-    uint8_t *sm = smem_raw + (c.base - raw);
-    c.bars = c.base + kOffBar;
-    volatile uint32_t *tmem_slot = (volatile uint32_t *)(sm + kOffBar + 16);
-    c.s_abort = (volatile int *)(sm + kOffBar + 20);
-    volatile int *s_item = (volatile int *)(sm + kOffBar + 24);
-    c.tid = threadIdx.x;
-    c.warp = c.tid >> 5;
-    c.lane = c.tid & 31;
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *sm = smem_raw + (base - raw);
+    const uint32_t bars = base + kOffBar;
+    volatile uint32_t *tmem_slot = (volatile uint32_t *)(sm + kOffBar + 8 * kNumBars);
+    volatile int *s_abort = (volatile int *)(sm + kOffBar + 8 * kNumBars + 4);
+    volatile int *s_item = (volatile int *)(sm + kOffBar + 8 * kNumBars + 8);  // [kSchedDepth]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    if (c.tid == 0) {
-        mbar_init(c.bars, 1);
-        mbar_init(c.bars + 8, 1);
-        *c.s_abort = 0;
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bars + 8 * (kBarRFull + i), kLoadWarps);
+            mbar_init(bars + 8 * (kBarREmpty + i), 1);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(bars + 8 * (kBarCFull + i), kLoadWarps);
+            mbar_init(bars + 8 * (kBarCEmpty + i), 1);
+        }
+        mbar_init(bars + 8 * kBarSFull, 1);
+        mbar_init(bars + 8 * kBarAFull, kComputeWarps);
+        mbar_init(bars + 8 * kBarGDone, 1);
+        mbar_init(bars + 8 * kBarFinal, 1);
+        for (int i = 0; i < kSchedDepth; ++i) {
+            mbar_init(bars + 8 * (kBarSchedFull + i), 1);
+            mbar_init(bars + 8 * (kBarSchedEmpty + i), kSchedReaders);
+        }
+        *s_abort = 0;
         fence_mbar_init();
     }
-    if (c.warp == 0) {
+    if (warp == kMmaWarp) {
         tmem_alloc(smem_u32((const void *)tmem_slot), 512);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    c.tmem = *tmem_slot;
+    const uint32_t tmem = *tmem_slot;
 
 #ifdef MATE_TRACE
     long long tr[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    c.tr = tr;
     const long long tr_start = clock64();
 #endif
-    uint32_t ph_s = 0, ph_fin = 0;
-    const int n_items = p.n_units * 4;
-    while (true) {
-        if (c.tid == 0) *s_item = atomicAdd(p.counter, 1);
-        __syncthreads();
-        const int item = *s_item;
-        __syncthreads();
-        if (item >= n_items || *c.s_abort) break;
-        const FwdUnit un = load_unit(p.units + (item >> 2));
-        const int h = item & 1;
-        if (item & 2) process_item<true>(p, c, un, h, ph_s, ph_fin);
-        else process_item<false>(p, c, un, h, ph_s, ph_fin);
+    // every wait is bounded; the first one to expire raises the abort flag, which ends all roles
+    auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+        for (uint32_t it = 0; it < kWaitLimit; ++it) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if (*s_abort) return false;
+        }
+        *s_abort = 1;
+        atomicOr(p.status + 1, 1);
+        return false;
+    };
+    // n-th entry of the item list of this CTA (-1 = exhausted); see the scheduler in the loader role
+    auto next_item = [&](uint32_t n) -> int {
+        const int slot = n % kSchedDepth;
+        if (!wait(bars + 8 * (kBarSchedFull + slot), (n / kSchedDepth) & 1)) return -1;
+        const int it = s_item[slot];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + 8 * (kBarSchedEmpty + slot));
+        return it;
+    };
+
+    if (warp < kComputeWarps) {
+        // ------------------------------------------------------------------ arithmetic + epilogue
+        const int r = tid & 127;   // row of the tile = lane of tensor memory
+        const int cq = warp >> 2;  // columns 32 cq .. 32 cq + 31 of a column tile
+        const uint32_t tm = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        uint32_t ph_s = 0, ph_g = 0, c_cnt = 0;
+        bool alive = true;
+
+        for (uint32_t n = 0; alive; ++n) {
+            const int it = next_item(n);
+            if (it < 0) break;
+            const Item x = make_item(p, it);
+            if (x.rows_h == 0) continue;
+            const FwdUnit &un = x.un;
+            const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
+            const int32_t *perm = vp.perm + (size_t)un.b * p.N;
+            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const bool row_valid = r < x.rows_h;
+            const int t_row = x.row0 + min(r, x.rows_h - 1);  // rows past the end shadow the last one
+            const int orig = perm[t_row];
+
+            if (x.n_tiles == 0) {  // padding rows: zero gradients
+                if (row_valid && cq == 0) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (!x.key_side) reinterpret_cast<uint4 *>(p.dQ + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
+                        if (x.key_side) {
+                            reinterpret_cast<uint4 *>(p.dK + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
+                            reinterpret_cast<uint4 *>(p.dV + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
+                        }
+                    }
+                }
+                continue;
+            }
+
+            // own segment of this row and the envelope over the 32 rows of the warp
+            int my_lo = 0, my_hi = 0, w_lo_min = 0, w_lo_max = 0, w_hi_min = 0, w_hi_max = 0;
+            if (x.n_tiles > x.nA) {
+                my_lo = vp.seg_lo[(size_t)un.b * p.N + t_row];
+                my_hi = vp.seg_hi[(size_t)un.b * p.N + t_row];
+                w_lo_min = w_lo_max = my_lo;
+                w_hi_min = w_hi_max = my_hi;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    w_lo_min = min(w_lo_min, __shfl_xor_sync(0xffffffffu, w_lo_min, o));
+                    w_lo_max = max(w_lo_max, __shfl_xor_sync(0xffffffffu, w_lo_max, o));
+                    w_hi_min = min(w_hi_min, __shfl_xor_sync(0xffffffffu, w_hi_min, o));
+                    w_hi_max = max(w_hi_max, __shfl_xor_sync(0xffffffffu, w_hi_max, o));
+                }
+            }
+            float row_lse2 = 0.f, row_D = 0.f;  // query side: this row's LSE (log2 domain) and D
+            if (!x.key_side) {
+                row_lse2 = p.LSE[bh + orig] * 1.4426950408889634f;
+                row_D = p.D[bh + orig];
+            }
+
+            // the tile loop is compiled once per side (the side is a compile-time constant inside)
+            auto tile_loop = [&](auto side) {
+            constexpr bool kKeySide = decltype(side)::value;
+            TileInfo t;
+            int c0 = 0, c1 = 0;
+            bool first = true;
+            for (int i = next_tile(x, 0, t, c0, c1); i < x.n_tiles && alive; i = next_tile(x, i + 1, t, c0, c1)) {
+                const int st = c_cnt % kStages;
+                ++c_cnt;
+                // this thread's columns [r_lo, r_hi) of the tile and the warp's envelope
+                int r_lo, r_hi, e_lo_min, e_lo_max, e_hi_min, e_hi_max;
+                if (!t.is_b) {
+                    r_lo = e_lo_min = e_lo_max = 0;
+                    r_hi = e_hi_min = e_hi_max = un.kA_end - t.k0;
+                } else {
+                    r_lo = my_lo - t.k0;
+                    r_hi = my_hi - t.k0;
+                    e_lo_min = w_lo_min - t.k0;
+                    e_lo_max = w_lo_max - t.k0;
+                    e_hi_min = w_hi_min - t.k0;
+                    e_hi_max = w_hi_max - t.k0;
+                }
+                const uint32_t r_span = (uint32_t)max(r_hi - r_lo, 0);
+                const float4 *vec4 = reinterpret_cast<const float4 *>(sm + kOffVec + st * 1024);
+
+                TR_T0(t_ws);
+                if (!(alive = wait(bars + 8 * kBarSFull, ph_s))) break;
+                ph_s ^= 1;
+                tc_fence_after();
+                TR_ADD(0, t_ws);
+                TR_T0(t_cmp);
+                bool a_free = first;  // the operand columns are free once the gradient MMAs of the previous tile are done
+#pragma unroll 1
+                for (int cc = 0; cc < 2 && alive; ++cc) {
+                    const int cb = cq * 32 + cc * 16;  // 16 columns at a time
+                    if (cb >= c1 || cb + 16 <= c0) continue;  // outside the columns the MMAs touch
+                    uint32_t pk_p[8], pk_ds[8];
+                    if (cb + 16 <= e_lo_min || cb >= e_hi_max) {
+                        // no row of the warp has a pair here
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) pk_p[e] = pk_ds[e] = 0u;
+                    } else {
+                        uint32_t sv[16], tv[16];
+                        TR_T0(t_ld);
+                        tmem_ld16(tm + kTmS + cb, sv);
+                        tmem_ld16(tm + kTmT + cb, tv);
+                        tc_wait_ld();
+                        TR_ADD(4, t_ld);
+                        const bool full = cb >= e_lo_max && cb + 16 <= e_hi_min;
+#pragma unroll
+                        for (int e = 0; e < 16; e += 4) {
+                            float lse2[4], Dv[4];
+                            if (kKeySide) {
+                                const float4 a = vec4[(cb + e) >> 2], d4 = vec4[32 + ((cb + e) >> 2)];
+                                lse2[0] = a.x; lse2[1] = a.y; lse2[2] = a.z; lse2[3] = a.w;
+                                Dv[0] = d4.x; Dv[1] = d4.y; Dv[2] = d4.z; Dv[3] = d4.w;
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    lse2[q] = row_lse2;
+                                    Dv[q] = row_D;
+                                }
+                            }
+                            float pv[4], dsv[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float xx = fmaf(__uint_as_float(sv[e + q]), p.scale_log2, -lse2[q]);
+                                pv[q] = ex2(xx);
+                                if (!full && (uint32_t)(cb + e + q - r_lo) >= r_span) pv[q] = 0.f;
+                                dsv[q] = pv[q] * (__uint_as_float(tv[e + q]) - Dv[q]);
+                            }
+                            pk_p[e >> 1] = pack_bf16(pv[0], pv[1]);
+                            pk_p[(e >> 1) + 1] = pack_bf16(pv[2], pv[3]);
+                            pk_ds[e >> 1] = pack_bf16(dsv[0], dsv[1]);
+                            pk_ds[(e >> 1) + 1] = pack_bf16(dsv[2], dsv[3]);
+                        }
+                    }
+                    if (!a_free) {
+                        TR_T0(t_wg);
+                        if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
+                        ph_g ^= 1;
+                        tc_fence_after();
+                        a_free = true;
+                        TR_ADD(1, t_wg);
+                    }
+                    if (kKeySide) {
+                        tmem_st8(tm + kTmA1 + (cb >> 1), pk_p);
+                        tmem_st8(tm + kTmA2 + (cb >> 1), pk_ds);
+                    } else {
+                        tmem_st8(tm + kTmA1 + (cb >> 1), pk_ds);
+                    }
+                }
+                if (!alive) break;
+                if (!a_free) {  // nothing written in this tile: the phase is consumed all the same
+                    if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
+                    ph_g ^= 1;
+                }
+                first = false;
+                TR_T0(t_sig);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bars + 8 * kBarAFull);
+                TR_ADD(6, t_sig);
+                TR_ADD(2, t_cmp);
+                TR_INC(7);
+            }
+            };
+            if (x.key_side) tile_loop(std::true_type{});
+            else tile_loop(std::false_type{});
+            if (!alive) break;
+
+            // epilogue: wait for the last gradient MMAs, then scatter the rows (or add split partial sums)
+            TR_T0(t_ep);
+            if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
+            ph_g ^= 1;
+            tc_fence_after();
+            if (x.key_side || cq < 2) {
+                // column quarters 0, 1: the two halves of accumulator 1 (dQ or dV); 2, 3 (key side): of accumulator 2 (dK)
+                const int half = cq & 1;
+                const uint32_t tacc = tm + (cq < 2 ? kTmAcc1 : kTmAcc2) + 32 * half;
+                const float mul = (!x.key_side || cq >= 2) ? p.scale : 1.f;
+                __nv_bfloat16 *out = !x.key_side ? p.dQ : (cq < 2 ? p.dV : p.dK);
+                const int plane = !x.key_side ? 0 : (cq < 2 ? 2 : 1);
+#pragma unroll 1
+                for (int sub = 0; sub < 2; ++sub) {
+                    uint32_t a0[16];
+                    tmem_ld16(tacc + 16 * sub, a0);
+                    tc_wait_ld();
+                    if (!row_valid) continue;
+                    if (un.n_parts == 1) {
+                        uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + 32 * half + 16 * sub);
+#pragma unroll
+                        for (int q = 0; q < 2; ++q) {
+                            const uint32_t *src = a0 + 8 * q;
+                            dst[q] = make_uint4(pack_bf16(__uint_as_float(src[0]) * mul, __uint_as_float(src[1]) * mul),
+                                                pack_bf16(__uint_as_float(src[2]) * mul, __uint_as_float(src[3]) * mul),
+                                                pack_bf16(__uint_as_float(src[4]) * mul, __uint_as_float(src[5]) * mul),
+                                                pack_bf16(__uint_as_float(src[6]) * mul, __uint_as_float(src[7]) * mul));
+                        }
+                    } else {
+                        // split prefix rows: view position = original position < P
+                        float *dst = p.acc32 + plane * p.plane + (((size_t)un.b * p.H + un.h) * p.P + orig) * 64 +
+                                     32 * half + 16 * sub;
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) atomicAdd(dst + e, __uint_as_float(a0[e]) * mul);
+                    }
+                }
+            }
+            tc_fence_before();  // the accumulators were read; the next item may overwrite them
+            TR_ADD(3, t_ep);
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer (one thread)
+        if (lane == 0) {
+            uint32_t c_cnt = 0, item_cnt = 0, ph_a = 0;
+            bool alive = true;
+            const uint32_t idesc_g = idesc_bf16(128, 64, 0, 1);  // B = 16 rows of the column tile x 64, MN-major
+            for (uint32_t n = 0; alive; ++n) {
+                const int slot = n % kSchedDepth;
+                if (!(alive = wait(bars + 8 * (kBarSchedFull + slot), (n / kSchedDepth) & 1))) break;
+                const int it = s_item[slot];
+                mbar_arrive(bars + 8 * (kBarSchedEmpty + slot));
+                if (it < 0) break;
+                const Item x = make_item(p, it);
+                if (x.rows_h == 0 || x.n_tiles == 0) continue;
+                const int rb = item_cnt & 1;
+                TR_T0(t_rf);
+                if (!(alive = wait(bars + 8 * (kBarRFull + rb), (item_cnt >> 1) & 1))) break;
+                tc_fence_after();
+                TR_ADD(0, t_rf);
+                const uint32_t ra = smem_desc_lo(base + kOffR + rb * 2 * kTileBytes), rbb = ra + (kTileBytes >> 4);
+
+                // gradient MMAs of the tile whose operands are (being) written: columns [g0, g1) of stage g_st
+                int g0 = 0, g1 = 0, g_st = 0;
+                bool have_g = false, acc = false;
+                auto issue_grad = [&]() {
+                    TR_T0(t_g);
+                    const uint32_t sCa = base + kOffC + g_st * 2 * kTileBytes;
+                    uint32_t a_lo = smem_desc_lo(sCa + g0 * kRowBytes), b_lo = a_lo + (kTileBytes >> 4);
+                    uint32_t tA1 = tmem + kTmA1 + (g0 >> 1), tA2 = tmem + kTmA2 + (g0 >> 1);
+                    const int n_ks = (g1 - g0) >> 4;
+                    constexpr uint32_t kStepLo = (16 * kRowBytes) >> 4;  // 16 rows of the column tile per step
+                    if (x.key_side) {
+                        mma_ts_lean_flag(tmem + kTmAcc1, tA1, b_lo, idesc_g, acc);  // dV += P^T dO
+                        mma_ts_lean_flag(tmem + kTmAcc2, tA2, a_lo, idesc_g, acc);  // dK += dS^T Q
+#pragma unroll 1
+                        for (int ks = 1; ks < n_ks; ++ks) {
+                            a_lo += kStepLo;
+                            b_lo += kStepLo;
+                            tA1 += 8;
+                            tA2 += 8;
+                            mma_ts_lean<1>(tmem + kTmAcc1, tA1, b_lo, idesc_g);
+                            mma_ts_lean<1>(tmem + kTmAcc2, tA2, a_lo, idesc_g);
+                        }
+                    } else {
+                        mma_ts_lean_flag(tmem + kTmAcc1, tA1, a_lo, idesc_g, acc);  // dQ += dS K
+#pragma unroll 1
+                        for (int ks = 1; ks < n_ks; ++ks) {
+                            a_lo += kStepLo;
+                            tA1 += 8;
+                            mma_ts_lean<1>(tmem + kTmAcc1, tA1, a_lo, idesc_g);
+                        }
+                    }
+                    acc = true;
+                    mma_commit(bars + 8 * kBarGDone);
+                    mma_commit(bars + 8 * (kBarCEmpty + g_st));
+                    TR_ADD(3, t_g);
+                };
+
+                TileInfo t;
+                int c0 = 0, c1 = 0;
+                for (int i = next_tile(x, 0, t, c0, c1); i < x.n_tiles && alive; i = next_tile(x, i + 1, t, c0, c1)) {
+                    const int st = c_cnt % kStages;
+                    TR_T0(t_cf);
+                    if (!(alive = wait(bars + 8 * (kBarCFull + st), (c_cnt / kStages) & 1))) break;
+                    TR_ADD(1, t_cf);
+                    ++c_cnt;
+                    if (have_g) {  // S and dP are free again once the arithmetic of the previous tile is done
+                        TR_T0(t_wa);
+                        if (!(alive = wait(bars + 8 * kBarAFull, ph_a))) break;
+                        ph_a ^= 1;
+                        TR_ADD(2, t_wa);
+                    }
+                    tc_fence_after();
+                    {
+                        TR_T0(t_s);
+                        const uint32_t idesc = idesc_bf16(128, c1 - c0, 0, 0);
+                        const uint32_t sCa = base + kOffC + st * 2 * kTileBytes;
+                        const uint32_t ca = smem_desc_lo(sCa + c0 * kRowBytes), cb = ca + (kTileBytes >> 4);
+                        mma_ss_lean<0>(tmem + kTmS + c0, ra, ca, idesc);  // S = Ra Ca^T, K = 64 as four steps of 16
+                        mma_ss_lean<1>(tmem + kTmS + c0, ra + 2, ca + 2, idesc);
+                        mma_ss_lean<1>(tmem + kTmS + c0, ra + 4, ca + 4, idesc);
+                        mma_ss_lean<1>(tmem + kTmS + c0, ra + 6, ca + 6, idesc);
+                        mma_ss_lean<0>(tmem + kTmT + c0, rbb, cb, idesc);  // dP = Rb Cb^T
+                        mma_ss_lean<1>(tmem + kTmT + c0, rbb + 2, cb + 2, idesc);
+                        mma_ss_lean<1>(tmem + kTmT + c0, rbb + 4, cb + 4, idesc);
+                        mma_ss_lean<1>(tmem + kTmT + c0, rbb + 6, cb + 6, idesc);
+                        mma_commit(bars + 8 * kBarSFull);
+                        TR_ADD(4, t_s);
+                        TR_INC(7);
+                    }
+                    if (have_g) issue_grad();  // of the previous tile, behind this tile's S and dP
+                    have_g = true;
+                    g0 = c0;
+                    g1 = c1;
+                    g_st = st;
+                }
+                if (!alive) break;
+                if (have_g) {
+                    if (!(alive = wait(bars + 8 * kBarAFull, ph_a))) break;
+                    ph_a ^= 1;
+                    tc_fence_after();
+                    issue_grad();
+                }
+                mma_commit(bars + 8 * (kBarREmpty + rb));
+                ++item_cnt;
+            }
+            // nothing of this CTA may still run on the tensor pipe when tensor memory is freed
+            mma_commit(bars + 8 * kBarFinal);
+            mbar_wait_bounded(bars + 8 * kBarFinal, 0, kWaitLimit);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ loaders
+        const int ltid = tid - 32 * kLoadWarp0;
+        uint32_t c_cnt = 0, item_cnt = 0;
+        uint32_t pend[kLag];
+#pragma unroll
+        for (int i = 0; i < kLag; ++i) pend[i] = 0;
+        bool alive = true;
+
+        // Commits the copies issued so far as one group and signals the barrier of the group that
+        // was committed kLag groups earlier (its copies have landed by then).
+        auto commit_and_signal = [&](uint32_t bar) {
+            cp_async_commit();
+            const uint32_t oldest = pend[0];
+#pragma unroll
+            for (int i = 0; i + 1 < kLag; ++i) pend[i] = pend[i + 1];
+            pend[kLag - 1] = bar;
+            if (oldest) {
+                cp_async_wait_group<kLag>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(oldest);
+            }
+        };
+        // Signals every group still pending.  Called before this warp blocks on a buffer that is
+        // not free yet: the consumers may need exactly those groups to free it.
+        auto flush = [&]() {
+            cp_async_wait_group<0>();
+            fence_proxy_async();
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < kLag; ++i) {
+                if (pend[i] && lane == 0) mbar_arrive(pend[i]);
+                pend[i] = 0;
+            }
+        };
+        auto wait_free = [&](uint32_t bar, uint32_t parity) -> bool {
+            if (__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) return true;
+            flush();
+            TR_T0(t_wf);
+            const bool ok = wait(bar, parity);
+            TR_ADD(0, t_wf);
+            return ok;
+        };
+
+        // scheduler (lane 0 of the first loader warp): the first item of a CTA is its own index,
+        // later ones come from the shared counter, each taken when the loaders are about to start on it
+        uint32_t produced = 0;
+        bool list_done = false;
+        const int n_items = p.n_units * 4;
+        auto produce = [&]() -> bool {
+            const int slot = produced % kSchedDepth;
+            if (produced >= (uint32_t)kSchedDepth &&
+                !wait(bars + 8 * (kBarSchedEmpty + slot), ((produced / kSchedDepth) & 1) ^ 1))
+                return false;
+            const int it = produced == 0 ? (int)blockIdx.x : atomicAdd(p.counter, 1) + (int)gridDim.x;
+            const int val = it < n_items ? it : -1;
+            s_item[slot] = val;
+            mbar_arrive(bars + 8 * (kBarSchedFull + slot));
+            ++produced;
+            if (val < 0) list_done = true;
+            return true;
+        };
+
+        for (uint32_t n = 0; alive; ++n) {
+            {   // before a loader warp blocks on the item list it signals its pending copy groups
+                const int slot = n % kSchedDepth;
+                bool must_wait;
+                if (warp == kLoadWarp0) {
+                    must_wait = produced >= (uint32_t)kSchedDepth &&
+                                !mbar_test_wait(bars + 8 * (kBarSchedEmpty + slot), ((produced / kSchedDepth) & 1) ^ 1);
+                    must_wait = __shfl_sync(0xffffffffu, (int)must_wait, 0) != 0;
+                } else {
+                    must_wait = !__all_sync(0xffffffffu, mbar_test_wait(bars + 8 * (kBarSchedFull + slot),
+                                                                       (n / kSchedDepth) & 1));
+                }
+                if (must_wait) flush();
+            }
+            if (ltid == 0) {
+                while (!list_done && produced <= n)
+                    if (!produce()) break;
+            }
+            __syncwarp();
+            const int it = next_item(n);
+            if (it < 0) break;
+            const Item x = make_item(p, it);
+            if (x.rows_h == 0 || x.n_tiles == 0) continue;
+            const FwdUnit &un = x.un;
+            const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
+            const int32_t *perm = vp.perm + (size_t)un.b * p.N;
+            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const __nv_bfloat16 *Ra_bh = (x.key_side ? p.K : p.Q) + bh * 64, *Rb_bh = (x.key_side ? p.V : p.dO) + bh * 64;
+            const __nv_bfloat16 *Ca_bh = (x.key_side ? p.Q : p.K) + bh * 64, *Cb_bh = (x.key_side ? p.dO : p.V) + bh * 64;
+
+            {   // row operands
+                const int rb = item_cnt & 1;
+                int idx[kPasses];
+                load_indices(idx, perm, x.row0, kTile, x.rows_h - 1, ltid);
+                if (!(alive = wait_free(bars + 8 * (kBarREmpty + rb), ((item_cnt >> 1) & 1) ^ 1))) break;
+                const uint32_t sRa = base + kOffR + rb * 2 * kTileBytes;
+                copy_pair(sRa, sRa + kTileBytes, Ra_bh, Rb_bh, idx, ltid);
+                commit_and_signal(bars + 8 * (kBarRFull + rb));
+                ++item_cnt;
+            }
+            TileInfo t;
+            int c0 = 0, c1 = 0;
+            for (int i = next_tile(x, 0, t, c0, c1); i < x.n_tiles; i = next_tile(x, i + 1, t, c0, c1)) {
+                const int st = c_cnt % kStages;
+                const int n16 = (t.w + 15) & ~15;
+                int idx[kPasses];
+                load_indices(idx, perm, t.k0, n16, t.w - 1, ltid);
+                float v_lse[2] = {0.f, 0.f}, v_D[2] = {0.f, 0.f};
+                if (x.key_side) {  // LSE (log2 domain) and D of the query columns
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const int cidx = ltid + q * kLoadThreads;
+                        if (cidx < kTile) {
+                            const int o = perm[t.k0 + min(cidx, t.w - 1)];
+                            v_lse[q] = p.LSE[bh + o] * 1.4426950408889634f;
+                            v_D[q] = p.D[bh + o];
+                        }
+                    }
+                }
+                if (!(alive = wait_free(bars + 8 * (kBarCEmpty + st), ((c_cnt / kStages) & 1) ^ 1))) break;
+                const uint32_t sCa = base + kOffC + st * 2 * kTileBytes;
+                copy_pair(sCa, sCa + kTileBytes, Ca_bh, Cb_bh, idx, ltid);
+                if (x.key_side) {
+                    float *vec = reinterpret_cast<float *>(sm + kOffVec + st * 1024);
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const int cidx = ltid + q * kLoadThreads;
+                        if (cidx < kTile) {
+                            vec[cidx] = v_lse[q];
+                            vec[128 + cidx] = v_D[q];
+                        }
+                    }
+                }
+                commit_and_signal(bars + 8 * (kBarCFull + st));
+                ++c_cnt;
+            }
+        }
+        flush();  // drain: signal the groups still pending
     }
 
 #ifdef MATE_TRACE
-    if (c.tid == 0 || c.tid == 255) {
-        long long *o = g_trace_bwd + blockIdx.x * 16 + (c.tid == 0 ? 0 : 8);
+    if (lane == 0 && (warp == 0 || warp == 4 || warp == kMmaWarp || warp == kLoadWarp0)) {
+        const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == kMmaWarp ? 2 : 3;
+        long long *o = g_trace_bwd + blockIdx.x * 32 + role * 8;
         for (int i = 0; i < 8; ++i) o[i] = tr[i];
-        if (c.tid == 0) o[6] = clock64() - tr_start;  // thread 0: total instead of the item sum
+        if (role == 0) o[5] = clock64() - tr_start;
     }
 #endif
-    // nothing of this CTA may still run on the tensor pipe when tensor memory is freed
-    if (*c.s_abort && c.tid == 0) {
-        mma_commit(c.bars + 8);
-        mbar_wait_bounded(c.bars + 8, ph_fin, kWaitLimit);
-    }
     tc_fence_before();
     __syncthreads();
-    if (c.warp == 0) tmem_dealloc(c.tmem, 512);
+    if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
 bool g_attr_set = false;
@@ -600,8 +834,8 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 }  // namespace mate
 
 #ifdef MATE_TRACE
-// copies the cycle counters of the last backward launch to the host: [148 CTAs][2 threads][8]
+// copies the cycle counters of the last backward launch to the host: [148 CTAs][4 roles][8]
 extern "C" int mate_debug_trace_bwd(long long *host_out) {
-    return cudaMemcpyFromSymbol(host_out, mate::g_trace_bwd, sizeof(long long) * 148 * 16) == cudaSuccess ? 0 : -4;
+    return cudaMemcpyFromSymbol(host_out, mate::g_trace_bwd, sizeof(long long) * 148 * 32) == cudaSuccess ? 0 : -4;
 }
 #endif
