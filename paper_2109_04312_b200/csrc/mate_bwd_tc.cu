@@ -18,8 +18,9 @@
 //               tile, the lane of tensor memory; each takes 32 of the 128 columns of a column tile.
 //               S and dP (fp32) come out of tensor memory, P / dS (bf16 pairs) go back into it as
 //               MMA operands.
-//   warp  16    one thread issues every tcgen05.mma: S and dP of tile n + 1 go ahead of the
-//               gradient MMAs of tile n, which then run under the arithmetic of tile n + 1
+//   warp  16    one thread issues every tcgen05.mma: S and dP of tile n + 1 are issued as soon as
+//               those of tile n sit in registers, ahead of the gradient MMAs of tile n, so both
+//               run under the arithmetic
 //   warps 17-19 loaders: gather rows by view-order index with 16-byte cp.async into 128-byte
 //               swizzled shared memory (row operands double buffered, column tiles in a ring of 3)
 // The gradients accumulate in tensor memory and are scattered to the rows' original positions in
@@ -68,7 +69,8 @@ enum {
     kBarFinal = 13,
     kBarSchedFull = 14,   // [kSchedDepth] scheduler -> every warp (count 1)
     kBarSchedEmpty = 18,  // [kSchedDepth] every warp -> scheduler (count kSchedReaders)
-    kNumBars = 22
+    kBarSTFree = 22,      // arithmetic -> MMA: S and dP of a tile are in registers (count: one per warp)
+    kNumBars = 23
 };
 constexpr int kSchedDepth = 4;
 constexpr int kSchedReaders = kComputeWarps + 1 + kLoadWarps;
@@ -252,6 +254,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
         }
         mbar_init(bars + 8 * kBarSFull, 1);
         mbar_init(bars + 8 * kBarAFull, kComputeWarps);
+        mbar_init(bars + 8 * kBarSTFree, kComputeWarps);
         mbar_init(bars + 8 * kBarGDone, 1);
         mbar_init(bars + 8 * kBarFinal, 1);
         for (int i = 0; i < kSchedDepth; ++i) {
@@ -382,6 +385,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                 TR_ADD(0, t_ws);
                 TR_T0(t_cmp);
                 bool a_free = first;  // the operand columns are free once the gradient MMAs of the previous tile are done
+                // S and dP may be overwritten as soon as this warp's last load of them has completed
+                const int cb1 = cq * 32 + 16;
+                const bool load1 = !(cb1 >= c1 || cb1 + 16 <= c0) && !(cb1 + 16 <= e_lo_min || cb1 >= e_hi_max);
+                bool st_signalled = false;
+                auto signal_st = [&]() {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bars + 8 * kBarSTFree);
+                    st_signalled = true;
+                };
 #pragma unroll 1
                 for (int cc = 0; cc < 2 && alive; ++cc) {
                     const int cb = cq * 32 + cc * 16;  // 16 columns at a time
@@ -398,6 +411,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                         tmem_ld16(tm + kTmT + cb, tv);
                         tc_wait_ld();
                         TR_ADD(4, t_ld);
+                        if (cc == 1 || !load1) signal_st();
                         const bool full = cb >= e_lo_max && cb + 16 <= e_hi_min;
 #pragma unroll
                         for (int e = 0; e < 16; e += 4) {
@@ -443,6 +457,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                     }
                 }
                 if (!alive) break;
+                if (!st_signalled) signal_st();
                 if (!a_free) {  // nothing written in this tile: the phase is consumed all the same
                     if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
                     ph_g ^= 1;
@@ -505,7 +520,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
     } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer (one thread)
         if (lane == 0) {
-            uint32_t c_cnt = 0, item_cnt = 0, ph_a = 0;
+            uint32_t c_cnt = 0, item_cnt = 0, ph_a = 0, ph_st = 0;
             bool alive = true;
             const uint32_t idesc_g = idesc_bf16(128, 64, 0, 1);  // B = 16 rows of the column tile x 64, MN-major
             for (uint32_t n = 0; alive; ++n) {
@@ -568,10 +583,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                     if (!(alive = wait(bars + 8 * (kBarCFull + st), (c_cnt / kStages) & 1))) break;
                     TR_ADD(1, t_cf);
                     ++c_cnt;
-                    if (have_g) {  // S and dP are free again once the arithmetic of the previous tile is done
+                    if (have_g) {  // S and dP are free again once the previous tile's values are in registers
                         TR_T0(t_wa);
-                        if (!(alive = wait(bars + 8 * kBarAFull, ph_a))) break;
-                        ph_a ^= 1;
+                        if (!(alive = wait(bars + 8 * kBarSTFree, ph_st))) break;
+                        ph_st ^= 1;
                         TR_ADD(2, t_wa);
                     }
                     tc_fence_after();
@@ -592,7 +607,14 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                         TR_ADD(4, t_s);
                         TR_INC(7);
                     }
-                    if (have_g) issue_grad();  // of the previous tile, behind this tile's S and dP
+                    if (have_g) {  // gradient MMAs of the previous tile, behind this tile's S and dP
+                        TR_T0(t_wa2);
+                        if (!(alive = wait(bars + 8 * kBarAFull, ph_a))) break;
+                        ph_a ^= 1;
+                        tc_fence_after();
+                        TR_ADD(5, t_wa2);
+                        issue_grad();
+                    }
                     have_g = true;
                     g0 = c0;
                     g1 = c1;
@@ -600,6 +622,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                 }
                 if (!alive) break;
                 if (have_g) {
+                    if (!(alive = wait(bars + 8 * kBarSTFree, ph_st))) break;
+                    ph_st ^= 1;
                     if (!(alive = wait(bars + 8 * kBarAFull, ph_a))) break;
                     ph_a ^= 1;
                     tc_fence_after();

@@ -117,14 +117,15 @@ __device__ __forceinline__ TileInfo tile_info(const FwdUnit &u, int i, int nA) {
 __device__ __forceinline__ int rows_of_half(const FwdUnit &u, int h) {
     return max(0, min(kTile, u.nq - h * kTile));
 }
-// Columns [c0, c1) of the tile (multiples of 16) that half h needs; c1 <= c0 when it skips the tile.
-__device__ __forceinline__ void half_cols(const FwdUnit &u, int h, const TileInfo &t, int &c0, int &c1) {
+// Columns [c0, c1) of the tile (multiples of 16) needed by a half whose rows' segments span keys
+// [lo, hi); c1 <= c0 when it skips the tile.
+__device__ __forceinline__ void half_cols(int lo, int hi, const TileInfo &t, int &c0, int &c1) {
     if (!t.is_b) {
         c0 = 0;
         c1 = (t.w + 15) & ~15;
     } else {
-        c0 = (max(u.lo[h], t.k0) - t.k0) & ~15;
-        c1 = (min(u.hi[h], t.k0 + t.w) - t.k0 + 15) & ~15;
+        c0 = (max(lo, t.k0) - t.k0) & ~15;
+        c1 = (min(hi, t.k0 + t.w) - t.k0 + 15) & ~15;
     }
 }
 
@@ -302,6 +303,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             const int t_row = un.q0 + h * kTile + min(r, rows_h - 1);  // rows past the end shadow the last one
             const int orig = perm[t_row];
             const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
+            const int h_lo = h ? un.lo[1] : un.lo[0], h_hi = h ? un.hi[1] : un.hi[0];  // segments of this half's rows
 
             if (n_tiles == 0) {  // padding rows: O = 0, LSE = -inf
                 if (row_valid) {
@@ -335,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             for (int i = 0; i < n_tiles && alive; ++i) {
                 const TileInfo t = tile_info(un, i, nA);
                 int c0, c1;
-                half_cols(un, h, t, c0, c1);
+                half_cols(h_lo, h_hi, t, c0, c1);
                 if (c1 <= c0) continue;
 
                 // this row's columns [r_lo, r_hi) and the warp's envelope, tile-local
@@ -559,6 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 if (u < 0) break;
                 const FwdUnit un = load_unit(p.units + u);
                 const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
+                const int h_lo = h ? un.lo[1] : un.lo[0], h_hi = h ? un.hi[1] : un.hi[0];  // segments of this half's rows
                 if (n_tiles == 0) continue;
                 const int qb = unit_cnt & 1;
                 TR_T0(t_qf);
@@ -611,7 +614,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     const int stage = c % kStages;
                     const uint32_t bar_kv = bars + 8 * (kBarKVFull + stage), par_kv = (c / kStages) & 1;
                     int c0 = 0, c1 = 0;
-                    if (has_rows) half_cols(un, h, t, c0, c1);
+                    if (has_rows) half_cols(h_lo, h_hi, t, c0, c1);
                     if (c1 <= c0) {  // this half skips the tile
                         if (wait_p) {  // nothing to issue ahead of the P V of the previous tile
                             if (!(alive = take_p())) break;
