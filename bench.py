@@ -57,7 +57,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -169,6 +169,17 @@ def run_reference(args, cfg):
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def reduce_over_ranks(times, work, world):
+    """Whole-job figures from per-rank ones: every rank runs its own replica (the path has no
+    exchange step), so the job's time is the slowest rank's (MAX) and its work the sum (SUM).
+    `times` and `work` are float64 tensors on the rank's device (CPU tensors under gloo)."""
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+        dist.all_reduce(work, op=dist.ReduceOp.SUM)
+    return times.tolist(), work.tolist()
 
 
 def run_mate(args, cfg):
@@ -288,11 +299,8 @@ def run_mate(args, cfg):
     times = torch.tensor([total_ms, float(np.median(fwd_ms)), float(np.median(bwd_ms)), e2e_ms,
                           float(fwd_ms.min()), float(bwd_ms.min())], dtype=torch.float64, device=dev)
     work = torch.tensor([pairs, n_valid_tokens], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-        dist.all_reduce(work, op=dist.ReduceOp.SUM)
-    total_ms, fwd_med, bwd_med, e2e_ms, fwd_min, bwd_min = times.tolist()
-    pairs_all, tokens_all = work.tolist()
+    (total_ms, fwd_med, bwd_med, e2e_ms, fwd_min, bwd_min), (pairs_all, tokens_all) = \
+        reduce_over_ranks(times, work, world)
     ff, fb = pair_flops(cfg, pairs_all)
     ms_per_step = total_ms / K
 
@@ -353,7 +361,7 @@ def run_mate(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="mate", choices=["mate", "reference"])
     ap.add_argument("--workload", default="long", choices=sorted(tables.CONFIGS))
