@@ -22,7 +22,7 @@
 //               those of tile n sit in registers, ahead of the gradient MMAs of tile n, so both
 //               run under the arithmetic
 //   warps 17-19 loaders: gather rows by view-order index with 16-byte cp.async into 128-byte
-//               swizzled shared memory (row operands double buffered, column tiles in a ring of 3)
+//               swizzled shared memory (row operands double buffered, column tiles in a ring of 4)
 // The gradients accumulate in tensor memory and are scattered to the rows' original positions in
 // the epilogue.
 #include <cuda_bf16.h>
@@ -48,7 +48,7 @@ constexpr int kLoadWarp0 = 17;
 constexpr int kLoadWarps = 3;
 constexpr int kLoadThreads = 32 * kLoadWarps;
 constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
-constexpr int kStages = 3;  // ring of column tiles
+constexpr int kStages = 4;  // ring of column tiles
 constexpr int kLag = 2;     // loader: copy groups in flight behind the newest one
 constexpr int kRowBytes = 128;
 constexpr int kTileBytes = kTile * kRowBytes;  // 16 KB
@@ -62,15 +62,15 @@ enum {
     kBarRFull = 0,    // [2] loaders -> MMA                  (count: loader warps)
     kBarREmpty = 2,   // [2] MMA commit -> loaders           (count 1)
     kBarCFull = 4,    // [kStages] loaders -> MMA            (count: loader warps)
-    kBarCEmpty = 7,   // [kStages] MMA commit -> loaders     (count 1)
-    kBarSFull = 10,   // MMA commit -> arithmetic: S and dP of a tile are complete (count 1)
-    kBarAFull = 11,   // arithmetic -> MMA: the bf16 operands of a tile are written (count: one per warp)
-    kBarGDone = 12,   // MMA commit -> arithmetic: the gradient MMAs of a tile are complete (count 1)
-    kBarFinal = 13,
-    kBarSchedFull = 14,   // [kSchedDepth] scheduler -> every warp (count 1)
-    kBarSchedEmpty = 18,  // [kSchedDepth] every warp -> scheduler (count kSchedReaders)
-    kBarSTFree = 22,      // arithmetic -> MMA: S and dP of a tile are in registers (count: one per warp)
-    kNumBars = 23
+    kBarCEmpty = 8,   // [kStages] MMA commit -> loaders     (count 1)
+    kBarSFull = 12,   // MMA commit -> arithmetic: S and dP of a tile are complete (count 1)
+    kBarAFull = 13,   // arithmetic -> MMA: the bf16 operands of a tile are written (count: one per warp)
+    kBarGDone = 14,   // MMA commit -> arithmetic: the gradient MMAs of a tile are complete (count 1)
+    kBarFinal = 15,
+    kBarSchedFull = 16,   // [kSchedDepth] scheduler -> every warp (count 1)
+    kBarSchedEmpty = 20,  // [kSchedDepth] every warp -> scheduler (count kSchedReaders)
+    kBarSTFree = 24,      // arithmetic -> MMA: S and dP of a tile are in registers (count: one per warp)
+    kNumBars = 25
 };
 constexpr int kSchedDepth = 4;
 constexpr int kSchedReaders = kComputeWarps + 1 + kLoadWarps;
