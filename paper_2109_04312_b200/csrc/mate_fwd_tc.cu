@@ -40,16 +40,16 @@ constexpr int kLoadWarp0 = 10;
 constexpr int kLoadWarps = 2;
 constexpr int kLoadThreads = 32 * kLoadWarps;
 constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
-constexpr int kStages = 3;                   // K/V ring
+constexpr int kStages = 5;                   // K/V ring
 constexpr int kLag = 2;                      // loader: copy groups in flight behind the newest one
 
 constexpr int kRowBytes = 128;                 // 64 bf16
 constexpr int kTileBytes = kTile * kRowBytes;  // 16 KB: 128 rows
 constexpr uint32_t kOffQ = 0;                                // [2 buffers][2 halves] x 16 KB
 constexpr uint32_t kOffKV = 4 * kTileBytes;                  // [kStages] x (K 16 KB, V 16 KB)
-constexpr uint32_t kOffP = kOffKV + kStages * 2 * kTileBytes;  // [2 halves] x 32 KB (two 64-column blocks)
-constexpr uint32_t kOffBar = kOffP + 4 * kTileBytes;
-constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;        // + slack for the 1024-byte alignment
+constexpr uint32_t kOffBar = kOffKV + kStages * 2 * kTileBytes;
+constexpr uint32_t kSmemBytes = kOffBar + 512 + 1024;        // + slack for the 1024-byte alignment
+static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 // tensor memory: S of half h at column 128 h; O at 256 + 64 h; P (bf16 pairs) at 384 + 64 h
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kTmemO = 256;
@@ -62,18 +62,18 @@ enum {
     kBarQFull = 0,    // [2] loader -> MMA         (count: loader warps)
     kBarQEmpty = 2,   // [2] MMA commit -> loader  (count 2: one per half)
     kBarKVFull = 4,   // [kStages] loader -> MMA   (count: loader warps)
-    kBarKVEmpty = 8,  // [kStages] MMA -> loader   (count 2: one per half)
-    kBarSFull = 12,   // [2] MMA commit -> softmax (count 1)
-    kBarPFull = 14,   // [2] softmax -> MMA        (count 4: one per warp)
-    kBarPVDone = 16,  // [2] MMA commit -> softmax: the P V of a tile is complete (count 1)
-    kBarFinal = 18,       // [2]
-    kBarSchedFull = 20,   // [kSchedDepth] scheduler -> every warp that follows the unit list (count 1)
-    kBarSchedEmpty = 24,  // [kSchedDepth] those warps -> scheduler (count kSchedReaders)
-    kNumBars = 28
+    kBarKVEmpty = 9,  // [kStages] MMA -> loader   (count 2: one per half)
+    kBarSFull = 14,   // [2] MMA commit -> softmax (count 1)
+    kBarPFull = 16,   // [2] softmax -> MMA        (count 4: one per warp)
+    kBarPVDone = 18,  // [2] MMA commit -> softmax: the P V of a tile is complete (count 1)
+    kBarFinal = 20,       // [2]
+    kBarSchedFull = 22,   // [kSchedDepth] scheduler -> every warp that follows the unit list (count 1)
+    kBarSchedEmpty = 26,  // [kSchedDepth] those warps -> scheduler (count kSchedReaders)
+    kNumBars = 30
 };
 constexpr int kSchedDepth = 4;
 constexpr int kSchedReaders = kSoftmaxWarps + kMmaWarps + kLoadWarps;
-static_assert(kStages <= 4, "barrier slots");
+static_assert(kStages <= 5, "barrier slots");
 
 struct Params {
     const __nv_bfloat16 *Q, *K, *V;
