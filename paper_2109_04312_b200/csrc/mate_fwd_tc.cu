@@ -10,9 +10,13 @@
 //               memory with 16-byte cp.async (the gather of Section 3.1 fused into the loads)
 //
 // Per key tile and half:   S = Q K^T  (tcgen05.mma, M = 128, N <= 128, K = 64, accumulator in TMEM)
-//                          online softmax in the exp2 domain: row max, P = exp2(S c - m), row sum
-//                          O += P V   (tcgen05.mma, M = 128, N = 64; O stays in TMEM and is
-//                          rescaled only when a row's running max grows by more than 2^8)
+//                          online softmax in the exp2 domain: P = exp2(S c - m), row sum.  After a
+//                          unit's first tile, P is formed in one pass over S with the running max m;
+//                          the tile's own max is tracked on the way and only a growth by more than
+//                          2^8 sends the tile through the two-pass path (max, rescale O, exp)
+//                          O += P V   (tcgen05.mma, M = 128, N = 64, P read from TMEM; O stays there)
+// S is released to the MMA issuer as soon as its last 32 columns sit in registers, so the Q K^T of
+// the half's next tile runs under the rest of the exponentials.
 // The two halves share every K/V tile and alternate on the tensor pipe, so the exponentials of
 // one half overlap the MMAs of the other.  Key tiles of range B are visited by a half only where
 // they meet the segments of its rows, and inside a tile a warp evaluates only the 32-column chunks
@@ -69,7 +73,8 @@ enum {
     kBarFinal = 20,       // [2]
     kBarSchedFull = 22,   // [kSchedDepth] scheduler -> every warp that follows the unit list (count 1)
     kBarSchedEmpty = 26,  // [kSchedDepth] those warps -> scheduler (count kSchedReaders)
-    kNumBars = 30
+    kBarSFree = 30,       // [2] softmax -> MMA: S of a tile has been read for the last time (count 4: one per warp)
+    kNumBars = 32
 };
 constexpr int kSchedDepth = 4;
 constexpr int kSchedReaders = kSoftmaxWarps + kMmaWarps + kLoadWarps;
@@ -224,6 +229,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             mbar_init(bars + 8 * (kBarSFull + i), 1);
             mbar_init(bars + 8 * (kBarPFull + i), 4);
             mbar_init(bars + 8 * (kBarPVDone + i), 1);
+            mbar_init(bars + 8 * (kBarSFree + i), 4);
         }
         for (int i = 0; i < kStages; ++i) {
             mbar_init(bars + 8 * (kBarKVFull + i), kLoadWarps);
@@ -283,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         const uint32_t tO = tmem + lane_base + kTmemO + h * 64;
         const uint32_t tP = tmem + lane_base + kTmemP + h * 64;
         const uint32_t bar_s = bars + 8 * (kBarSFull + h), bar_p = bars + 8 * (kBarPFull + h),
-                       bar_pv = bars + 8 * (kBarPVDone + h);
+                       bar_pv = bars + 8 * (kBarPVDone + h), bar_sf = bars + 8 * (kBarSFree + h);
         uint32_t ph_s = 0, ph_pv = 0;
         bool alive = true;
 
@@ -361,72 +367,127 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 ph_s ^= 1;
                 tc_fence_after();
                 TR_ADD(0, t_ws);
-                TR_T0(t_p1);
-
-                // pass 1: row max of the raw scores, 32 columns at a time (chunks in which no row of
-                // the warp has a key are not looked at)
-                float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-                for (int ch = ch0; ch < ch1; ++ch) {
-                    const int cb = ch * 32;
-                    if (cb + 32 <= e_lo_min || cb >= e_hi_max) continue;
-                    uint32_t v[32];
-                    tmem_ld32(tS + cb, v);
-                    tc_wait_ld();
-                    chunk_max(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, tm);
-                }
-                TR_ADD(2, t_p1);
-                const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
-                const float t2 = tmax * p.scale_log2;
-                const bool grow = t2 > m2 + kRescaleThreshold;  // also true for the first finite max
-                float alpha = 1.f;
-                if (grow) {
-                    alpha = ex2(m2 - t2);  // 0 when m2 = -inf
-                    m2 = t2;
-                    l *= alpha;
-                }
+                // last chunk of the tile that this warp reads from tensor memory (-1: none): after it,
+                // S may be overwritten
+                int last_ld = -1;
+                for (int ch = ch0; ch < ch1; ++ch)
+                    if (!(ch * 32 + 32 <= e_lo_min || ch * 32 >= e_hi_max)) last_ld = ch;
+                auto release_s = [&]() {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_sf);
+                };
                 // P of the previous tile is still being read, and O written, until that tile's P V is done
-                if (!first) {
+                bool pv_waited = first;
+                auto wait_pv = [&]() -> bool {
+                    if (pv_waited) return true;
                     TR_T0(t_wpv);
-                    if (!(alive = wait(bar_pv, ph_pv))) break;
+                    if (!(alive = wait(bar_pv, ph_pv))) return false;
                     ph_pv ^= 1;
                     tc_fence_after();
+                    pv_waited = true;
                     TR_ADD(1, t_wpv);
-                }
-                if (!first && __any_sync(0xffffffffu, grow)) {
-#pragma unroll
-                    for (int c2 = 0; c2 < 2; ++c2) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + c2 * 32, o);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tmem_st32(tO + c2 * 32, o);
-                    }
-                    tc_wait_st();
-                }
-                const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
+                    return true;
+                };
 
-                // pass 2: P = exp2(s * scale_log2 - m) as bf16 pairs into the P columns, row sum
+                bool two_pass = first;
                 TR_T0(t_p2);
-                float lsum = 0.f, lsum1 = 0.f;
+                if (!two_pass) {
+                    // one pass with the running max; the tile's own max is known before S is given up
+                    float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
+                    float lsum = 0.f, lsum1 = 0.f;
+                    bool redo = false;
 #pragma unroll 1
-                for (int ch = ch0; ch < ch1; ++ch) {
-                    const int cb = ch * 32;
-                    uint32_t packed[16];
-                    if (cb + 32 <= e_lo_min || cb >= e_hi_max) {
+                    for (int ch = ch0; ch < ch1; ++ch) {
+                        const int cb = ch * 32;
+                        uint32_t packed[16];
+                        if (cb + 32 <= e_lo_min || cb >= e_hi_max) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) packed[e] = 0u;
-                    } else {
+                            for (int e = 0; e < 16; ++e) packed[e] = 0u;
+                        } else {
+                            uint32_t v[32];
+                            tmem_ld32(tS + cb, v);
+                            tc_wait_ld();
+                            const bool full = cb >= e_lo_max && cb + 32 <= e_hi_min;
+                            chunk_max(v, cb, full, r_lo, r_span, tm);
+                            if (ch == last_ld) {
+                                const float t2 = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
+                                redo = __any_sync(0xffffffffu, t2 > m2 + kRescaleThreshold);
+                                if (redo) break;
+                                release_s();
+                            }
+                            chunk_exp(v, cb, full, r_lo, r_span, p.scale_log2, neg_m, packed, lsum, lsum1);
+                        }
+                        if (!wait_pv()) break;
+                        tmem_st16(tP + ch * 16, packed);
+                    }
+                    if (!alive) break;
+                    if (!redo) {
+                        if (last_ld < 0) release_s();
+                        l += lsum + lsum1;
+                    }
+                    two_pass = redo;
+                }
+                if (two_pass) {
+                    // pass 1: row max of the raw scores, 32 columns at a time (chunks in which no row of
+                    // the warp has a key are not looked at)
+                    float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+                    for (int ch = ch0; ch < ch1; ++ch) {
+                        const int cb = ch * 32;
+                        if (cb + 32 <= e_lo_min || cb >= e_hi_max) continue;
                         uint32_t v[32];
                         tmem_ld32(tS + cb, v);
                         tc_wait_ld();
-                        chunk_exp(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, p.scale_log2, neg_m,
-                                  packed, lsum, lsum1);
+                        chunk_max(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, tm);
                     }
-                    tmem_st16(tP + ch * 16, packed);
+                    const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
+                    const float t2 = tmax * p.scale_log2;
+                    const bool grow = t2 > m2 + kRescaleThreshold;  // also true for the first finite max
+                    float alpha = 1.f;
+                    if (grow) {
+                        alpha = ex2(m2 - t2);  // 0 when m2 = -inf
+                        m2 = t2;
+                        l *= alpha;
+                    }
+                    if (!wait_pv()) break;
+                    if (!first && __any_sync(0xffffffffu, grow)) {
+#pragma unroll
+                        for (int c2 = 0; c2 < 2; ++c2) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c2 * 32, o);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(tO + c2 * 32, o);
+                        }
+                        tc_wait_st();
+                    }
+                    const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
+
+                    // pass 2: P = exp2(s * scale_log2 - m) as bf16 pairs into the P columns, row sum
+                    float lsum = 0.f, lsum1 = 0.f;
+                    if (last_ld < 0) release_s();
+#pragma unroll 1
+                    for (int ch = ch0; ch < ch1; ++ch) {
+                        const int cb = ch * 32;
+                        uint32_t packed[16];
+                        if (cb + 32 <= e_lo_min || cb >= e_hi_max) {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) packed[e] = 0u;
+                        } else {
+                            uint32_t v[32];
+                            tmem_ld32(tS + cb, v);
+                            tc_wait_ld();
+                            if (ch == last_ld) release_s();
+                            chunk_exp(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, p.scale_log2, neg_m,
+                                      packed, lsum, lsum1);
+                        }
+                        tmem_st16(tP + ch * 16, packed);
+                    }
+                    l += lsum + lsum1;
                 }
-                l += lsum + lsum1;
                 first = false;
 
                 tc_wait_st();
@@ -546,12 +607,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
         // tile the half skips, by a plain arrival once the tile has landed.
         if (lane == 0) {
             const int h = warp - kMmaWarp;
-            uint32_t kv_cnt = 0, unit_cnt = 0, ph_p = 0;
+            uint32_t kv_cnt = 0, unit_cnt = 0, ph_p = 0, ph_sf = 0;
             bool alive = true;
             const uint32_t idesc_pv = idesc_bf16(128, 64, 0, 1);
             const uint32_t tSh0 = tmem + h * kTile, tOh = tmem + kTmemO + h * 64, tPh0 = tmem + kTmemP + h * 64;
             const uint32_t bar_p = bars + 8 * (kBarPFull + h), bar_s = bars + 8 * (kBarSFull + h),
-                           bar_pv = bars + 8 * (kBarPVDone + h);
+                           bar_pv = bars + 8 * (kBarPVDone + h), bar_sf = bars + 8 * (kBarSFree + h);
 
             for (uint32_t n = 0; alive; ++n) {
                 const int slot = n % kSchedDepth;
@@ -571,15 +632,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 const uint32_t q_lo = smem_desc_lo(base + kOffQ + (qb * 2 + h) * kTileBytes);
                 const bool has_rows = rows_of_half(un, h) > 0;
 
-                int qk_c0 = 0, qk_c1 = 0, qk_stage = 0;  // Q K^T issued, P not seen yet
-                int pv_c0 = 0, pv_c1 = 0, pv_stage = 0;  // P seen, P V not issued yet
-                bool wait_p = false, have_p = false, acc = false;
+                // `out`: a tile whose Q K^T has been issued and whose P V has not
+                int o_c0 = 0, o_c1 = 0, o_stage = 0;
+                bool out = false, acc = false;
 
-                auto issue_pv = [&]() {
+                auto issue_pv = [&]() -> bool {  // waits for the P of the outstanding tile, then O += P V
+                    TR_T0(t_wp);
+                    if (!wait(bar_p, ph_p)) return false;
+                    TR_ADD(1, t_wp);
+                    ph_p ^= 1;
+                    tc_fence_after();
                     TR_T0(t_pv);
-                    const int ks0 = pv_c0 >> 4, n_ks = (pv_c1 - pv_c0) >> 4;
+                    const int ks0 = o_c0 >> 4, n_ks = (o_c1 - o_c0) >> 4;
                     // V rows 16 ks .. 16 ks + 15 (2 KB per step), P columns 8 ks .. 8 ks + 7
-                    uint32_t v_lo = smem_desc_lo(base + kOffKV + pv_stage * 2 * kTileBytes + kTileBytes + ks0 * 16 * kRowBytes);
+                    uint32_t v_lo = smem_desc_lo(base + kOffKV + o_stage * 2 * kTileBytes + kTileBytes + ks0 * 16 * kRowBytes);
                     uint32_t tPh = tPh0 + ks0 * 8;
                     mma_ts_lean_flag(tOh, tPh, v_lo, idesc_pv, acc);
 #pragma unroll 1
@@ -589,22 +655,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         mma_ts_lean<1>(tOh, tPh, v_lo, idesc_pv);
                     }
                     acc = true;
-                    have_p = false;
+                    out = false;
                     mma_commit(bar_pv);
-                    mma_commit(bars + 8 * (kBarKVEmpty + pv_stage));
+                    mma_commit(bars + 8 * (kBarKVEmpty + o_stage));
                     TR_ADD(3, t_pv);
+                    return true;
                 };
-                auto take_p = [&]() -> bool {  // waits for the P of the outstanding Q K^T
-                    TR_T0(t_wp);
-                    if (!wait(bar_p, ph_p)) return false;
-                    TR_ADD(1, t_wp);
-                    ph_p ^= 1;
-                    tc_fence_after();
-                    wait_p = false;
-                    have_p = true;
-                    pv_c0 = qk_c0;
-                    pv_c1 = qk_c1;
-                    pv_stage = qk_stage;
+                auto wait_s_free = [&]() -> bool {  // S of the outstanding tile has been read for the last time
+                    TR_T0(t_sf);
+                    if (!wait(bar_sf, ph_sf)) return false;
+                    ph_sf ^= 1;
+                    TR_ADD(6, t_sf);
                     return true;
                 };
 
@@ -616,9 +677,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     int c0 = 0, c1 = 0;
                     if (has_rows) half_cols(h_lo, h_hi, t, c0, c1);
                     if (c1 <= c0) {  // this half skips the tile
-                        if (wait_p) {  // nothing to issue ahead of the P V of the previous tile
-                            if (!(alive = take_p())) break;
-                            issue_pv();
+                        if (out) {  // nothing to issue ahead of the P V of the outstanding tile
+                            if (!(alive = wait_s_free())) break;
+                            if (!(alive = issue_pv())) break;
                         }
                         TR_T0(t_kv);
                         if (!(alive = wait(bar_kv, par_kv))) break;
@@ -626,8 +687,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         mbar_arrive(bars + 8 * (kBarKVEmpty + stage));
                         continue;
                     }
-                    if (wait_p && !(alive = take_p())) break;
-                    if (have_p && !mbar_test_wait(bar_kv, par_kv)) issue_pv();  // the next tile is not there yet
+                    if (out && !(alive = wait_s_free())) break;
+                    if (out && !mbar_test_wait(bar_kv, par_kv)) {  // the next tile is not there yet
+                        if (!(alive = issue_pv())) break;
+                    }
                     TR_T0(t_kv);
                     if (!(alive = wait(bar_kv, par_kv))) break;
                     TR_ADD(5, t_kv);
@@ -642,17 +705,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         mma_ss_lean<1>(tSh, q_lo + 4, k_lo + 4, idesc);
                         mma_ss_lean<1>(tSh, q_lo + 6, k_lo + 6, idesc);
                         mma_commit(bar_s);
-                        wait_p = true;
-                        qk_c0 = c0;
-                        qk_c1 = c1;
-                        qk_stage = stage;
                         TR_ADD(2, t_qk);
                         TR_INC(4);
                     }
-                    if (have_p) issue_pv();
+                    if (out && !(alive = issue_pv())) break;  // P V of the previous tile, behind this tile's Q K^T
+                    out = true;
+                    o_c0 = c0;
+                    o_c1 = c1;
+                    o_stage = stage;
                 }
-                if (alive && wait_p) {
-                    if ((alive = take_p())) issue_pv();
+                if (alive && out) {
+                    if ((alive = wait_s_free())) alive = issue_pv();
                 }
                 kv_cnt += n_tiles;
                 if (!alive) break;
