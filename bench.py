@@ -206,9 +206,7 @@ def run_mate(args, cfg):
     plan = mate.mate_plan(torch.from_numpy(rows).to(dev), torch.from_numpy(cols).to(dev), cfg.P, hv,
                           cfg.n_rows, cfg.n_cols)
     pairs = float(plan.useful_pairs().sum())
-    _, bwd_ws = mate.mate_attn_workspace_bytes(plan, cfg.d, 0 if cfg.dtype == "bf16" else 1)
-    d_bytes = 256 + (cfg.B * cfg.H * N * 4 + 255) // 256 * 256
-    launches_per_step = 4 if bwd_ws > d_bytes else 3
+    launches_per_step = 3  # tc_fwd_kernel, rowdot_kernel, tc_bwd_kernel
     n_valid_tokens = float(sum(info["n_valid"]))
     f_fwd, f_bwd = pair_flops(cfg, pairs)
 
@@ -310,8 +308,8 @@ def run_mate(args, cfg):
         bwd_tflops = fb / (bwd_med * 1e-3) / 1e12
         # Roofline of the dominant kernel, tc_bwd_kernel (one launch = the whole backward of one
         # rank).  Its duration is taken as that of the mate_attn_bwd call, which also holds the
-        # small row-dot and rounding kernels (about 10% by the ncu launch list), so `achieved` is
-        # a lower bound for the kernel itself.
+        # small row-dot kernel (about 5% by the ncu launch list), so `achieved` is a lower bound
+        # for the kernel itself.
         fwd_tflops_rank = f_fwd / (float(np.mean(fwd_ms)) * 1e-3) / 1e12
         bwd_tflops_rank = f_bwd / (float(np.mean(bwd_ms)) * 1e-3) / 1e12
         line = {
@@ -339,8 +337,6 @@ def run_mate(args, cfg):
                              "traffic": NCU_TRAFFIC_BYTES["tc_fwd_kernel"]},
             "e2e": {"value": (ff + fb) / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            # per step: tc_fwd_kernel, rowdot_kernel, tc_bwd_kernel and, when prefix units are split,
-            # finalize_kernel
             "gpu_launches": K * launches_per_step,
             "clocks": sampler.summary(t_wall0, t_wall1),
         }

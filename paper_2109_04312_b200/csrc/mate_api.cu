@@ -82,119 +82,126 @@ int64_t half_cost(const FwdUnit &u, int h, const int32_t *so, int S) {
     return c;
 }
 
-int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_off_host) {
+// Units of all (example, head) pairs.  share = 0: no unit is split (the backward's list: its work
+// items are halves of units per side, fine enough as they are).  share > 0 (a CTA's share of the
+// total cost): a prefix-row unit, whose columns are all valid positions, that costs more than 1.3
+// shares is cut along the columns into parts of about 0.75 shares, to be combined in the kernel.
+void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_off_host, int64_t share,
+                std::vector<UnitCost> &all, int *n_slots, size_t *ws_bytes, int64_t *total_cost) {
     const int P = pl->P, N = pl->N;
-    std::vector<UnitCost> all;
-    // pass 1: units without splitting, to learn the total cost; pass 2 splits the long prefix units
-    int64_t split_tiles = 1 << 30;
-    for (int pass = 0; pass < 2; ++pass) {
-        all.clear();
-        pl->n_fwd_slots = 0;
-        pl->fwd_ws_bytes = 0;
-        int64_t total = 0;
-        for (int v = 0; v < 2; ++v) {
-            const ViewPlan &vp = pl->view[v];
-            if (vp.n_heads == 0) continue;
-            const int S = vp.max_id + 2;
-            for (int b = 0; b < pl->B; ++b) {
-                const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
-                const int nv = pl->n_valid[b];
-                auto seg_of = [&](int t) { return (int)(std::upper_bound(so, so + S, t) - so) - 1; };
-                std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
-                for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
-                    FwdUnit u{};
-                    u.q0 = q0;
-                    u.nq = std::min(mate::kUnitRows, P - q0);
-                    const int n_tiles = ceil_div(nv, kTile);
-                    const int want = ceil_div(n_tiles, (int)std::min<int64_t>(split_tiles, n_tiles));
-                    const int per = ceil_div(n_tiles, want);
-                    const int n_parts = ceil_div(n_tiles, per);  // every part holds at least one tile
-                    for (int part = 0; part < n_parts; ++part) {
-                        FwdUnit w = u;
-                        w.kA0 = part * per * kTile;
-                        w.kA_end = std::min(nv, (part + 1) * per * kTile);
-                        if (w.kA_end <= w.kA0) continue;
-                        w.n_parts = n_parts;
-                        w.part = part;
-                        proto.push_back({w, 0});
-                    }
+    all.clear();
+    *n_slots = 0;
+    *ws_bytes = 0;
+    *total_cost = 0;
+    for (int v = 0; v < 2; ++v) {
+        const ViewPlan &vp = pl->view[v];
+        if (vp.n_heads == 0) continue;
+        const int S = vp.max_id + 2;
+        for (int b = 0; b < pl->B; ++b) {
+            const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
+            const int nv = pl->n_valid[b];
+            auto seg_of = [&](int t) { return (int)(std::upper_bound(so, so + S, t) - so) - 1; };
+            std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
+            for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
+                FwdUnit u{};
+                u.q0 = q0;
+                u.nq = std::min(mate::kUnitRows, P - q0);
+                u.kA_end = nv;
+                const int n_tiles = ceil_div(nv, kTile);
+                const int64_t whole = half_cost(u, 0, so, S) + half_cost(u, 1, so, S);
+                int want = 1;
+                if (share > 0 && 10 * whole > 13 * share)
+                    want = (int)std::min<int64_t>(n_tiles, (4 * whole + 3 * share - 1) / (3 * share));
+                const int per = ceil_div(n_tiles, want);
+                const int n_parts = ceil_div(n_tiles, per);  // every part holds at least one tile
+                for (int part = 0; part < n_parts; ++part) {
+                    FwdUnit w = u;
+                    w.kA0 = part * per * kTile;
+                    w.kA_end = std::min(nv, (part + 1) * per * kTile);
+                    w.n_parts = n_parts;
+                    w.part = part;
+                    proto.push_back({w, 0});
                 }
-                for (int q0 = P; q0 < nv; q0 += mate::kUnitRows) {  // table rows: prefix + own segments
-                    FwdUnit u{};
-                    u.q0 = q0;
-                    u.nq = std::min(mate::kUnitRows, nv - q0);
-                    u.kA0 = 0;
-                    u.kA_end = P;
-                    u.kB0 = so[seg_of(q0)];
-                    u.kB_end = so[seg_of(q0 + u.nq - 1) + 1];
-                    for (int h = 0; h < 2; ++h) {
-                        const int r0 = q0 + h * kTile, r1 = std::min(q0 + u.nq, r0 + kTile) - 1;
-                        if (r1 < r0) continue;
-                        u.lo[h] = so[seg_of(r0)];
-                        u.hi[h] = so[seg_of(r1) + 1];
-                    }
-                    u.n_parts = 1;
-                    proto.push_back({u, 0});
+            }
+            for (int q0 = P; q0 < nv; q0 += mate::kUnitRows) {  // table rows: prefix + own segments
+                FwdUnit u{};
+                u.q0 = q0;
+                u.nq = std::min(mate::kUnitRows, nv - q0);
+                u.kA0 = 0;
+                u.kA_end = P;
+                u.kB0 = so[seg_of(q0)];
+                u.kB_end = so[seg_of(q0 + u.nq - 1) + 1];
+                for (int h = 0; h < 2; ++h) {
+                    const int r0 = q0 + h * kTile, r1 = std::min(q0 + u.nq, r0 + kTile) - 1;
+                    if (r1 < r0) continue;
+                    u.lo[h] = so[seg_of(r0)];
+                    u.hi[h] = so[seg_of(r1) + 1];
                 }
-                for (int q0 = nv; q0 < N; q0 += mate::kUnitRows) {  // padding rows: no key at all
-                    FwdUnit u{};
-                    u.q0 = q0;
-                    u.nq = std::min(mate::kUnitRows, N - q0);
-                    u.n_parts = 1;
-                    proto.push_back({u, 0});
-                }
-                for (auto &pc : proto) pc.cost = half_cost(pc.u, 0, so, S) + half_cost(pc.u, 1, so, S);
-                for (int h = 0; h < pl->H; ++h) {
-                    if (pl->head_view[h] != v) continue;
-                    int slot = -1;
-                    for (UnitCost pc : proto) {
-                        pc.u.b = b;
-                        pc.u.h = h;
-                        pc.u.ctr = -1;
-                        if (pc.u.n_parts > 1) {
-                            if (pc.u.part == 0) {
-                                slot = pl->n_fwd_slots++;
-                            }
-                            pc.u.ctr = slot;
-                            pc.u.ws_off = (int32_t)((pl->fwd_ws_bytes + pc.u.part * mate::kPartialBytes) >> 10);
-                            if (pc.u.part == pc.u.n_parts - 1) pl->fwd_ws_bytes += pc.u.n_parts * mate::kPartialBytes;
-                        }
-                        total += pc.cost;
-                        all.push_back(pc);
+                u.n_parts = 1;
+                proto.push_back({u, 0});
+            }
+            for (int q0 = nv; q0 < N; q0 += mate::kUnitRows) {  // padding rows: no key at all
+                FwdUnit u{};
+                u.q0 = q0;
+                u.nq = std::min(mate::kUnitRows, N - q0);
+                u.n_parts = 1;
+                proto.push_back({u, 0});
+            }
+            for (auto &pc : proto) pc.cost = half_cost(pc.u, 0, so, S) + half_cost(pc.u, 1, so, S);
+            for (int h = 0; h < pl->H; ++h) {
+                if (pl->head_view[h] != v) continue;
+                int slot = -1;
+                for (UnitCost pc : proto) {
+                    pc.u.b = b;
+                    pc.u.h = h;
+                    pc.u.ctr = -1;
+                    if (pc.u.n_parts > 1) {
+                        if (pc.u.part == 0) slot = (*n_slots)++;
+                        pc.u.ctr = slot;
+                        pc.u.ws_off = (int32_t)((*ws_bytes + pc.u.part * mate::kPartialBytes) >> 10);
+                        if (pc.u.part == pc.u.n_parts - 1) *ws_bytes += pc.u.n_parts * mate::kPartialBytes;
                     }
+                    *total_cost += pc.cost;
+                    all.push_back(pc);
                 }
             }
         }
-        if (pass == 0) {
-            // a split part should cost about half of a CTA's share (never below two key tiles)
-            const int64_t share = total / std::max(pl->n_ctas, 1);
-            const int64_t part_cost = std::max<int64_t>(share / 2, 1);
-            // cost of one key tile of a full prefix unit: 8 warps x 4 chunks
-            split_tiles = std::max<int64_t>(2, part_cost / 32);
-        }
     }
-    static_assert(mate::kPartialBytes % 1024 == 0, "ws_off counts KiB");
-
-    // longest first: the CTAs of the persistent kernel take units from the head of this list as
-    // they become free (a shared counter), so the order is the whole schedule
+    // longest first: the CTAs of the persistent kernels take work from the head of the list as they
+    // become free (a shared counter), so the order is the whole schedule
     std::stable_sort(all.begin(), all.end(), [](const UnitCost &a, const UnitCost &b) { return a.cost > b.cost; });
+}
+
+int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_off_host) {
+    static_assert(mate::kPartialBytes % 1024 == 0, "ws_off counts KiB");
     const int n_ctas = std::max(pl->n_ctas, 1);
-    pl->fwd_units.clear();
+    std::vector<UnitCost> all;
+    int n_slots = 0;
+    size_t ws_bytes = 0;
     int64_t total_cost = 0;
-    for (const UnitCost &uc : all) {
-        pl->fwd_units.push_back(uc.u);
-        total_cost += uc.cost;
-    }
+    // backward: unsplit list; its total cost also gives the share of a CTA
+    make_units(pl, seg_off_host, 0, all, &n_slots, &ws_bytes, &total_cost);
+    pl->bwd_units.clear();
+    for (const UnitCost &uc : all) pl->bwd_units.push_back(uc.u);
+    pl->n_bwd_units = (int)pl->bwd_units.size();
+    const int64_t share = std::max<int64_t>(total_cost / n_ctas, 1);
+    // forward: long prefix units split
+    make_units(pl, seg_off_host, share, all, &n_slots, &ws_bytes, &total_cost);
+    pl->fwd_units.clear();
+    for (const UnitCost &uc : all) pl->fwd_units.push_back(uc.u);
     pl->n_fwd_units = (int)pl->fwd_units.size();
+    pl->n_fwd_slots = n_slots;
+    pl->fwd_ws_bytes = ws_bytes;
     if (getenv("MATE_LOG"))
-        fprintf(stderr, "[mate] forward work-list: %d units, %d split slots, %d CTAs, cost total %lld (%.1f per CTA, "
-                        "largest unit %lld), split at %lld key tiles, workspace %zu bytes\n",
-                pl->n_fwd_units, pl->n_fwd_slots, n_ctas, (long long)total_cost, (double)total_cost / n_ctas,
-                all.empty() ? 0ll : (long long)all.front().cost, (long long)split_tiles, pl->fwd_ws_bytes);
+        fprintf(stderr, "[mate] work-lists: forward %d units (%d split), backward %d units, %d CTAs, cost total %lld "
+                        "(%.1f per CTA, largest forward unit %lld), forward workspace %zu bytes\n",
+                pl->n_fwd_units, pl->n_fwd_slots, pl->n_bwd_units, n_ctas, (long long)total_cost,
+                (double)total_cost / n_ctas, all.empty() ? 0ll : (long long)all.front().cost, pl->fwd_ws_bytes);
 
     // device copy: units, CTA offsets, arrival counters (zeroed once; the kernel resets them)
     Carver c(nullptr);
     c.take<FwdUnit>(pl->n_fwd_units);
+    c.take<FwdUnit>(pl->n_bwd_units);
     c.take<int32_t>(mate::kSchedWords + 8 * (size_t)pl->n_fwd_slots);
     const size_t bytes = align_up(c.off, 256);
     if (cudaMalloc(&pl->work_block, bytes) != cudaSuccess) {
@@ -203,6 +210,7 @@ int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
     }
     Carver d((char *)pl->work_block);
     pl->fwd_units_dev = d.take<FwdUnit>(pl->n_fwd_units);
+    pl->bwd_units_dev = d.take<FwdUnit>(pl->n_bwd_units);
     pl->fwd_counters_dev = d.take<int32_t>(mate::kSchedWords + 8 * (size_t)pl->n_fwd_slots);
     return MATE_OK;
 }
@@ -326,6 +334,9 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
                               sizeof(int32_t) * (mate::kSchedWords + 8 * (size_t)pl->n_fwd_slots), st) == cudaSuccess;
     if (pl->n_fwd_units > 0)
         up = up && cudaMemcpyAsync(pl->fwd_units_dev, pl->fwd_units.data(), sizeof(FwdUnit) * pl->n_fwd_units,
+                                   cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (pl->n_bwd_units > 0)
+        up = up && cudaMemcpyAsync(pl->bwd_units_dev, pl->bwd_units.data(), sizeof(FwdUnit) * pl->n_bwd_units,
                                    cudaMemcpyHostToDevice, st) == cudaSuccess;
     up = up && cudaStreamSynchronize(st) == cudaSuccess;
     if (!up) {

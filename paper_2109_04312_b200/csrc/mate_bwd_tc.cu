@@ -9,8 +9,7 @@
 //   query side  rows = queries, columns = their keys:  S = Q K^T, dP = dO V^T -> dS -> dQ += dS K
 //   key side    rows = keys, columns = the queries that attend them:  S^T = K Q^T, dP^T = V dO^T
 //               -> P^T, dS^T -> dV += P^T dO, dK += dS^T Q
-// so no gradient is accumulated across CTAs except for prefix rows whose column range was split
-// at plan time; those add fp32 partial sums into a scratch buffer that a last small kernel rounds.
+// so no gradient is accumulated across CTAs (the backward's list splits no unit).
 //
 // One persistent, warp-specialised CTA per SM (20 warps); work items (unit, half, side) are handed
 // out through a counter in the order of the plan's unit list.
@@ -82,8 +81,6 @@ struct Params {
     const __nv_bfloat16 *Q, *K, *V, *dO;
     const float *LSE, *D;  // [B, H, N], original order
     __nv_bfloat16 *dQ, *dK, *dV;
-    float *acc32;          // [3][B, H, P, 64] partial sums of split prefix rows (dQ, dK, dV)
-    size_t plane;          // floats per plane of acc32
     ViewPlan rowv, colv;
     const uint8_t *head_view;
     const FwdUnit *units;
@@ -181,26 +178,6 @@ __global__ void __launch_bounds__(256) rowdot_kernel(const __nv_bfloat16 *__rest
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) D[r] = acc;
-}
-
-// Rounds the fp32 sums of the split prefix rows into the outputs: blocks (u, y) cover unit u in
-// gridDim.y slices of rows; only the first part of a split unit does anything.  The rows of such a unit are prefix rows, whose view
-// position is their original position.
-__global__ void __launch_bounds__(256) finalize_kernel(const Params p) {
-    const FwdUnit un = load_unit(p.units + blockIdx.x);
-    if (un.n_parts <= 1 || un.part != 0) return;
-    const size_t bh = (size_t)un.b * p.H + un.h;
-    for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < un.nq * 32; i += blockDim.x * gridDim.y) {
-        const int row = un.q0 + (i >> 5), c2 = i & 31;
-        const float *a = p.acc32 + (bh * p.P + row) * 64 + 2 * c2;
-        const size_t dst = (bh * p.N + row) * 64 + 2 * c2;
-        const float2 q = *reinterpret_cast<const float2 *>(a);
-        const float2 k = *reinterpret_cast<const float2 *>(a + p.plane);
-        const float2 v = *reinterpret_cast<const float2 *>(a + 2 * p.plane);
-        *reinterpret_cast<__nv_bfloat162 *>(p.dQ + dst) = __floats2bfloat162_rn(q.x, q.y);
-        *reinterpret_cast<__nv_bfloat162 *>(p.dK + dst) = __floats2bfloat162_rn(k.x, k.y);
-        *reinterpret_cast<__nv_bfloat162 *>(p.dV + dst) = __floats2bfloat162_rn(v.x, v.y);
-    }
 }
 
 // Everything an item needs that does not depend on the role of the warp.
@@ -477,7 +454,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
             else tile_loop(std::false_type{});
             if (!alive) break;
 
-            // epilogue: wait for the last gradient MMAs, then scatter the rows (or add split partial sums)
+            // epilogue: wait for the last gradient MMAs, then scatter the rows to their original positions
             TR_T0(t_ep);
             if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
             ph_g ^= 1;
@@ -488,29 +465,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                 const uint32_t tacc = tm + (cq < 2 ? kTmAcc1 : kTmAcc2) + 32 * half;
                 const float mul = (!x.key_side || cq >= 2) ? p.scale : 1.f;
                 __nv_bfloat16 *out = !x.key_side ? p.dQ : (cq < 2 ? p.dV : p.dK);
-                const int plane = !x.key_side ? 0 : (cq < 2 ? 2 : 1);
 #pragma unroll 1
                 for (int sub = 0; sub < 2; ++sub) {
                     uint32_t a0[16];
                     tmem_ld16(tacc + 16 * sub, a0);
                     tc_wait_ld();
                     if (!row_valid) continue;
-                    if (un.n_parts == 1) {
-                        uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + 32 * half + 16 * sub);
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + 32 * half + 16 * sub);
 #pragma unroll
-                        for (int q = 0; q < 2; ++q) {
-                            const uint32_t *src = a0 + 8 * q;
-                            dst[q] = make_uint4(pack_bf16(__uint_as_float(src[0]) * mul, __uint_as_float(src[1]) * mul),
-                                                pack_bf16(__uint_as_float(src[2]) * mul, __uint_as_float(src[3]) * mul),
-                                                pack_bf16(__uint_as_float(src[4]) * mul, __uint_as_float(src[5]) * mul),
-                                                pack_bf16(__uint_as_float(src[6]) * mul, __uint_as_float(src[7]) * mul));
-                        }
-                    } else {
-                        // split prefix rows: view position = original position < P
-                        float *dst = p.acc32 + plane * p.plane + (((size_t)un.b * p.H + un.h) * p.P + orig) * 64 +
-                                     32 * half + 16 * sub;
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) atomicAdd(dst + e, __uint_as_float(a0[e]) * mul);
+                    for (int q = 0; q < 2; ++q) {
+                        const uint32_t *src = a0 + 8 * q;
+                        dst[q] = make_uint4(pack_bf16(__uint_as_float(src[0]) * mul, __uint_as_float(src[1]) * mul),
+                                            pack_bf16(__uint_as_float(src[2]) * mul, __uint_as_float(src[3]) * mul),
+                                            pack_bf16(__uint_as_float(src[4]) * mul, __uint_as_float(src[5]) * mul),
+                                            pack_bf16(__uint_as_float(src[6]) * mul, __uint_as_float(src[7]) * mul));
                     }
                 }
             }
@@ -800,18 +768,15 @@ inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 }  // namespace
 
-// workspace: [256 B counters][D: B*H*N floats][acc32: 3 planes of B*H*P*64 floats, only with split units]
+// workspace: [256 B counters][D: B*H*N floats]
 size_t tc_bwd_workspace(const mate_plan_t *plan) {
-    const size_t bhn = (size_t)plan->B * plan->H * plan->N;
-    size_t bytes = 256 + align256(bhn * sizeof(float));
-    if (plan->n_fwd_slots > 0) bytes += align256(3 * (size_t)plan->B * plan->H * plan->P * 64 * sizeof(float));
-    return bytes;
+    return 256 + align256((size_t)plan->B * plan->H * plan->N * sizeof(float));
 }
 
 int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, const void *O,
            const float *LSE, const void *dO, float scale, void *dQ, void *dK, void *dV, void *workspace,
            cudaStream_t stream) {
-    if (plan->n_fwd_units == 0) return MATE_OK;
+    if (plan->n_bwd_units == 0) return MATE_OK;
     if (!g_attr_set) {
         if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kSmemBytes) != cudaSuccess)
@@ -832,13 +797,11 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.dQ = (__nv_bfloat16 *)dQ;
     p.dK = (__nv_bfloat16 *)dK;
     p.dV = (__nv_bfloat16 *)dV;
-    p.plane = (size_t)plan->B * plan->H * plan->P * 64;
-    p.acc32 = plan->n_fwd_slots > 0 ? (float *)(ws + 256 + align256(bhn * sizeof(float))) : nullptr;
     p.rowv = plan->view[0];
     p.colv = plan->view[1];
     p.head_view = plan->head_view_dev;
-    p.units = plan->fwd_units_dev;
-    p.n_units = plan->n_fwd_units;
+    p.units = plan->bwd_units_dev;
+    p.n_units = plan->n_bwd_units;
     p.N = plan->N;
     p.H = plan->H;
     p.P = plan->P;
@@ -847,11 +810,8 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.status = plan->status_dev;
 
     if (cudaMemsetAsync(ws, 0, 256, stream) != cudaSuccess) return MATE_ERR_CUDA;
-    if (p.acc32 && cudaMemsetAsync(p.acc32, 0, 3 * p.plane * sizeof(float), stream) != cudaSuccess)
-        return MATE_ERR_CUDA;
     rowdot_kernel<<<(unsigned)((bhn + 7) / 8), 256, 0, stream>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, D, bhn);
     tc_bwd_kernel<<<plan->n_ctas, kThreads, kSmemBytes, stream>>>(p);
-    if (p.acc32) finalize_kernel<<<dim3(plan->n_fwd_units, 16), 256, 0, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 

@@ -73,6 +73,10 @@ struct mate_plan_s {
     int n_ctas = 0;                       // CTAs of the persistent kernel (SMs of the plan's device)
     size_t fwd_ws_bytes = 0;              // partial results of the split units
     std::vector<mate::FwdUnit> fwd_units; // host copy
+    // tensor-core backward work-list: the same units with no prefix unit split
+    mate::FwdUnit *bwd_units_dev = nullptr;
+    int n_bwd_units = 0;
+    std::vector<mate::FwdUnit> bwd_units;
 };
 
 namespace mate {
