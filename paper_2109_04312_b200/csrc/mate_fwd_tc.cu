@@ -688,9 +688,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         continue;
                     }
                     if (out && !(alive = wait_s_free())) break;
-                    if (out && !mbar_test_wait(bar_kv, par_kv)) {  // the next tile is not there yet
-                        if (!(alive = issue_pv())) break;
-                    }
                     TR_T0(t_kv);
                     if (!(alive = wait(bar_kv, par_kv))) break;
                     TR_ADD(5, t_kv);
