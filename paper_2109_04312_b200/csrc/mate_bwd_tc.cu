@@ -11,16 +11,16 @@
 //               -> P^T, dS^T -> dV += P^T dO, dK += dS^T Q
 // so no gradient is accumulated across CTAs (the backward's list splits no unit).
 //
-// One persistent, warp-specialised CTA per SM (20 warps); work items (unit, half, side) are handed
+// One persistent, warp-specialised CTA per SM (12 warps); work items (unit, half, side) are handed
 // out through a counter in the order of the plan's unit list.
-//   warps 0-15  arithmetic: four threads (r, r + 128, r + 256, r + 384) share row r of the 128-row
-//               tile, the lane of tensor memory; each takes 32 of the 128 columns of a column tile.
+//   warps 0-7   arithmetic: two threads (r, r + 128) share row r of the 128-row tile, the lane of
+//               tensor memory; each takes 64 of the 128 columns of a column tile, 32 at a time.
 //               S and dP (fp32) come out of tensor memory, P / dS (bf16 pairs) go back into it as
-//               MMA operands.
-//   warp  16    one thread issues every tcgen05.mma: S and dP of tile n + 1 are issued as soon as
+//               MMA operands.  (Sixteen warps with 32 columns each were measured 3% slower.)
+//   warp  8     one thread issues every tcgen05.mma: S and dP of tile n + 1 are issued as soon as
 //               those of tile n sit in registers, ahead of the gradient MMAs of tile n, so both
 //               run under the arithmetic
-//   warps 17-19 loaders: gather rows by view-order index with 16-byte cp.async into 128-byte
+//   warps 9-11  loaders: gather rows by view-order index with 16-byte cp.async into 128-byte
 //               swizzled shared memory (row operands double buffered, column tiles in a ring of 4)
 // The gradients accumulate in tensor memory and are scattered to the rows' original positions in
 // the epilogue.
@@ -41,9 +41,12 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kComputeWarps = 16;
-constexpr int kMmaWarp = 16;
-constexpr int kLoadWarp0 = 17;
+constexpr int kComputeWarps = 8;                       // 4 per group of 32 columns-per-thread
+constexpr int kColsPerThread = 128 / (kComputeWarps / 4);  // columns of a tile per arithmetic thread
+constexpr int kRound = 32;                             // columns worked on at a time (16 or 32)
+constexpr int kRounds = kColsPerThread / kRound;
+constexpr int kMmaWarp = kComputeWarps;
+constexpr int kLoadWarp0 = kComputeWarps + 1;
 constexpr int kLoadWarps = 3;
 constexpr int kLoadThreads = 32 * kLoadWarps;
 constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
@@ -159,6 +162,12 @@ __device__ __forceinline__ void copy_pair(uint32_t s_a, uint32_t s_b, const __nv
         }
     }
 }
+
+// tensor-memory access of one round of columns, by array size
+[[maybe_unused]] __device__ __forceinline__ void tmem_ld_round(uint32_t taddr, uint32_t (&v)[16]) { tmem_ld16(taddr, v); }
+__device__ __forceinline__ void tmem_ld_round(uint32_t taddr, uint32_t (&v)[32]) { tmem_ld32(taddr, v); }
+[[maybe_unused]] __device__ __forceinline__ void tmem_st_round(uint32_t taddr, const uint32_t (&v)[8]) { tmem_st8(taddr, v); }
+__device__ __forceinline__ void tmem_st_round(uint32_t taddr, const uint32_t (&v)[16]) { tmem_st16(taddr, v); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
@@ -277,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
     if (warp < kComputeWarps) {
         // ------------------------------------------------------------------ arithmetic + epilogue
         const int r = tid & 127;   // row of the tile = lane of tensor memory
-        const int cq = warp >> 2;  // columns 32 cq .. 32 cq + 31 of a column tile
+        const int cq = warp >> 2;  // columns kColsPerThread * cq .. + kColsPerThread - 1 of a column tile
         const uint32_t tm = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t ph_s = 0, ph_g = 0, c_cnt = 0;
         bool alive = true;
@@ -363,8 +372,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                 TR_T0(t_cmp);
                 bool a_free = first;  // the operand columns are free once the gradient MMAs of the previous tile are done
                 // S and dP may be overwritten as soon as this warp's last load of them has completed
-                const int cb1 = cq * 32 + 16;
-                const bool load1 = !(cb1 >= c1 || cb1 + 16 <= c0) && !(cb1 + 16 <= e_lo_min || cb1 >= e_hi_max);
+                int last_ld = -1;  // last round of this warp that reads tensor memory
+#pragma unroll
+                for (int cc = 0; cc < kRounds; ++cc) {
+                    const int cbx = cq * kColsPerThread + cc * kRound;
+                    if (!(cbx >= c1 || cbx + kRound <= c0) && !(cbx + kRound <= e_lo_min || cbx >= e_hi_max)) last_ld = cc;
+                }
                 bool st_signalled = false;
                 auto signal_st = [&]() {
                     tc_fence_before();
@@ -373,25 +386,25 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                     st_signalled = true;
                 };
 #pragma unroll 1
-                for (int cc = 0; cc < 2 && alive; ++cc) {
-                    const int cb = cq * 32 + cc * 16;  // 16 columns at a time
-                    if (cb >= c1 || cb + 16 <= c0) continue;  // outside the columns the MMAs touch
-                    uint32_t pk_p[8], pk_ds[8];
-                    if (cb + 16 <= e_lo_min || cb >= e_hi_max) {
+                for (int cc = 0; cc < kRounds && alive; ++cc) {
+                    const int cb = cq * kColsPerThread + cc * kRound;  // kRound columns at a time
+                    if (cb >= c1 || cb + kRound <= c0) continue;  // outside the columns the MMAs touch
+                    uint32_t pk_p[kRound / 2], pk_ds[kRound / 2];
+                    if (cb + kRound <= e_lo_min || cb >= e_hi_max) {
                         // no row of the warp has a pair here
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) pk_p[e] = pk_ds[e] = 0u;
+                        for (int e = 0; e < kRound / 2; ++e) pk_p[e] = pk_ds[e] = 0u;
                     } else {
-                        uint32_t sv[16], tv[16];
+                        uint32_t sv[kRound], tv[kRound];
                         TR_T0(t_ld);
-                        tmem_ld16(tm + kTmS + cb, sv);
-                        tmem_ld16(tm + kTmT + cb, tv);
+                        tmem_ld_round(tm + kTmS + cb, sv);
+                        tmem_ld_round(tm + kTmT + cb, tv);
                         tc_wait_ld();
                         TR_ADD(4, t_ld);
-                        if (cc == 1 || !load1) signal_st();
-                        const bool full = cb >= e_lo_max && cb + 16 <= e_hi_min;
+                        if (cc == last_ld) signal_st();
+                        const bool full = cb >= e_lo_max && cb + kRound <= e_hi_min;
 #pragma unroll
-                        for (int e = 0; e < 16; e += 4) {
+                        for (int e = 0; e < kRound; e += 4) {
                             float lse2[4], Dv[4];
                             if (kKeySide) {
                                 const float4 a = vec4[(cb + e) >> 2], d4 = vec4[32 + ((cb + e) >> 2)];
@@ -426,12 +439,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                         a_free = true;
                         TR_ADD(1, t_wg);
                     }
-                    if (kKeySide) {
-                        tmem_st8(tm + kTmA1 + (cb >> 1), pk_p);
-                        tmem_st8(tm + kTmA2 + (cb >> 1), pk_ds);
-                    } else {
-                        tmem_st8(tm + kTmA1 + (cb >> 1), pk_ds);
-                    }
+                    if (kKeySide) tmem_st_round(tm + kTmA1 + (cb >> 1), pk_p);
+                    tmem_st_round(tm + (kKeySide ? kTmA2 : kTmA1) + (cb >> 1), pk_ds);
                 }
                 if (!alive) break;
                 if (!st_signalled) signal_st();
@@ -459,19 +468,23 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
             if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
             ph_g ^= 1;
             tc_fence_after();
-            if (x.key_side || cq < 2) {
-                // column quarters 0, 1: the two halves of accumulator 1 (dQ or dV); 2, 3 (key side): of accumulator 2 (dK)
-                const int half = cq & 1;
-                const uint32_t tacc = tm + (cq < 2 ? kTmAcc1 : kTmAcc2) + 32 * half;
-                const float mul = (!x.key_side || cq >= 2) ? p.scale : 1.f;
-                __nv_bfloat16 *out = !x.key_side ? p.dQ : (cq < 2 ? p.dV : p.dK);
+            {
+                // The accumulator columns (dQ: 64; key side: dV | dK = 128) are shared out evenly among
+                // the column groups of the arithmetic warps, 16 columns at a time.
+                constexpr int kGroups = kComputeWarps / 4;
+                const int n_cols = (x.key_side ? 128 : 64) / kGroups;
 #pragma unroll 1
-                for (int sub = 0; sub < 2; ++sub) {
+                for (int sub = 0; sub < n_cols / 16; ++sub) {
+                    const int cacc = cq * n_cols + 16 * sub;
+                    const bool second = cacc >= 64;  // dK
+                    const int col = second ? cacc - 64 : cacc;
                     uint32_t a0[16];
-                    tmem_ld16(tacc + 16 * sub, a0);
+                    tmem_ld16(tm + (second ? kTmAcc2 : kTmAcc1) + col, a0);
                     tc_wait_ld();
                     if (!row_valid) continue;
-                    uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + 32 * half + 16 * sub);
+                    const float mul = (!x.key_side || second) ? p.scale : 1.f;
+                    __nv_bfloat16 *out = !x.key_side ? p.dQ : (second ? p.dK : p.dV);
+                    uint4 *dst = reinterpret_cast<uint4 *>(out + (bh + orig) * 64 + col);
 #pragma unroll
                     for (int q = 0; q < 2; ++q) {
                         const uint32_t *src = a0 + 8 * q;
