@@ -81,6 +81,21 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
               const uint8_t *head_view, int H, int max_row_id, int max_col_id, void *stream,
               mate_plan_t **out);
 
+/* The same plan for the bucketed, approximate form of the pattern (Section 3.1 and Appendix D: a
+ * global section G, which here is the prefix, and a local section cut into buckets of R positions
+ * of each head's own order; the paper uses R = 42).  In a head's order the positions behind the
+ * prefix form buckets of `radius` consecutive positions; a table token attends the prefix and,
+ * of its own row / column, only the keys in its own bucket and the two adjacent ones.  Prefix
+ * tokens still attend every non-padding position.  The order (perm, inv_perm, seg_off) is that
+ * of mate_plan; only the key ranges, the work-lists and the pair counts differ.  The pattern
+ * stays symmetric, so the forward and the backward calls take such a plan unchanged.  A radius
+ * at least as long as the longest row / column segment gives back the exact pattern, as the
+ * paper notes; radius = 0 means exactly that (mate_plan); radius < 0 is MATE_ERR_INVALID_ARG.
+ * All other arguments, ownership and errors as for mate_plan. */
+int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len,
+                       const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
+                       void *stream, mate_plan_t **out);
+
 /* Copies one view's order to HOST arrays (any pointer may be null to skip it):
  *   perm      int32 [B, N]          perm[b][t] = original position of the t-th token of the view
  *   inv_perm  int32 [B, N]          inverse of perm

@@ -40,6 +40,8 @@ def _load():
     lib.mate_status_string.argtypes = [i32]
     lib.mate_plan.restype = i32
     lib.mate_plan.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, vp, C.POINTER(vp)]
+    lib.mate_plan_bucketed.restype = i32
+    lib.mate_plan_bucketed.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_get.restype = i32
     lib.mate_plan_get.argtypes = [vp, i32, vp, vp, vp]
     lib.mate_plan_useful_pairs.restype = i32
@@ -129,7 +131,12 @@ class Plan:
             pass
 
 
-def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_id=None) -> Plan:
+def mate_plan_bucketed(row_ids, col_ids, prefix_len, head_view, radius, max_row_id=None, max_col_id=None) -> Plan:
+    """Plan of the bucketed variant (see mate_plan_bucketed in mate.h); radius = 0 is the exact pattern."""
+    return mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id, max_col_id, radius=radius)
+
+
+def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_id=None, radius=0) -> Plan:
     """row_ids, col_ids: int32 CUDA tensors [B, N]; head_view: sequence of 0 (row) / 1 (column)."""
     if row_ids.dtype != torch.int32 or col_ids.dtype != torch.int32 or row_ids.shape != col_ids.shape \
             or row_ids.dim() != 2:
@@ -142,7 +149,14 @@ def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_
         max_col_id = max(int(col_ids.max().item()), 0)
     handle = C.c_void_p()
     with torch.cuda.device(row_ids.device):
-        _check(_load().mate_plan(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N,
+        lib = _load()
+        if radius:
+            _check(lib.mate_plan_bucketed(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N,
+                                          int(prefix_len), hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
+                                          int(max_col_id), int(radius), _stream(), C.byref(handle)),
+                   "mate_plan_bucketed")
+        else:
+            _check(lib.mate_plan(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N,
                                  int(prefix_len), hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
                                  int(max_col_id), _stream(), C.byref(handle)), "mate_plan")
     return Plan(handle, B, N, int(prefix_len), int(hv.shape[0]), int(max_row_id), int(max_col_id),

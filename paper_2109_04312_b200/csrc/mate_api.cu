@@ -64,19 +64,37 @@ struct UnitCost {
     int64_t cost;
 };
 
-int64_t half_cost(const FwdUnit &u, int h, const int32_t *so, int S) {
+// Column range of one table row (view position t) of one (example, view): its segment, clipped to the
+// three adjacent buckets when the plan is bucketed.  The same arithmetic as step 4 of the plan kernel.
+struct RowBounds {
+    const int32_t *so;
+    int S, P, radius;
+    int seg_of(int t) const { return (int)(std::upper_bound(so, so + S, t) - so) - 1; }
+    int lo(int t) const {
+        const int l = so[seg_of(t)];
+        if (radius <= 0) return l;
+        const int64_t bk = (t - P) / radius;
+        return (int)std::max<int64_t>(l, P + (bk - 1) * radius);
+    }
+    int hi(int t) const {
+        const int h = so[seg_of(t) + 1];
+        if (radius <= 0) return h;
+        const int64_t bk = (t - P) / radius;
+        return (int)std::min<int64_t>(h, P + (bk + 2) * radius);
+    }
+};
+
+int64_t half_cost(const FwdUnit &u, int h, const RowBounds &rb) {
     const int rows = std::min(kTile, u.nq - h * kTile);
     if (rows <= 0) return 0;
     int64_t c = kCostPerHalf;
     const int n_warps = ceil_div(rows, 32);
     c += (int64_t)n_warps * ceil_div(std::max(u.kA_end - u.kA0, 0), kChunk);
     if (u.kB_end > u.kB0) {
-        auto seg_of = [&](int t) { return (int)(std::upper_bound(so, so + S, t) - so) - 1; };
         for (int w = 0; w < n_warps; ++w) {
             const int t0 = u.q0 + h * kTile + w * 32;
             const int t1 = std::min(t0 + 32, u.q0 + h * kTile + rows) - 1;
-            const int lo = so[seg_of(t0)], hi = so[seg_of(t1) + 1];
-            c += ceil_div(hi - lo, kChunk) + 1;  // + 1: chunks are aligned to the tile, not to lo
+            c += ceil_div(rb.hi(t1) - rb.lo(t0), kChunk) + 1;  // + 1: chunks are aligned to the tile, not to lo
         }
     }
     return c;
@@ -100,7 +118,7 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
         for (int b = 0; b < pl->B; ++b) {
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
             const int nv = pl->n_valid[b];
-            auto seg_of = [&](int t) { return (int)(std::upper_bound(so, so + S, t) - so) - 1; };
+            const RowBounds rb{so, S, P, pl->radius};
             std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
             for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
                 FwdUnit u{};
@@ -108,7 +126,7 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
                 u.nq = std::min(mate::kUnitRows, P - q0);
                 u.kA_end = nv;
                 const int n_tiles = ceil_div(nv, kTile);
-                const int64_t whole = half_cost(u, 0, so, S) + half_cost(u, 1, so, S);
+                const int64_t whole = half_cost(u, 0, rb) + half_cost(u, 1, rb);
                 int want = 1;
                 if (share > 0 && 10 * whole > 13 * share)
                     want = (int)std::min<int64_t>(n_tiles, (4 * whole + 3 * share - 1) / (3 * share));
@@ -129,13 +147,13 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
                 u.nq = std::min(mate::kUnitRows, nv - q0);
                 u.kA0 = 0;
                 u.kA_end = P;
-                u.kB0 = so[seg_of(q0)];
-                u.kB_end = so[seg_of(q0 + u.nq - 1) + 1];
+                u.kB0 = rb.lo(q0);   // lo and hi do not decrease along the rows
+                u.kB_end = rb.hi(q0 + u.nq - 1);
                 for (int h = 0; h < 2; ++h) {
                     const int r0 = q0 + h * kTile, r1 = std::min(q0 + u.nq, r0 + kTile) - 1;
                     if (r1 < r0) continue;
-                    u.lo[h] = so[seg_of(r0)];
-                    u.hi[h] = so[seg_of(r1) + 1];
+                    u.lo[h] = rb.lo(r0);
+                    u.hi[h] = rb.hi(r1);
                 }
                 u.n_parts = 1;
                 proto.push_back({u, 0});
@@ -147,7 +165,7 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
                 u.n_parts = 1;
                 proto.push_back({u, 0});
             }
-            for (auto &pc : proto) pc.cost = half_cost(pc.u, 0, so, S) + half_cost(pc.u, 1, so, S);
+            for (auto &pc : proto) pc.cost = half_cost(pc.u, 0, rb) + half_cost(pc.u, 1, rb);
             for (int h = 0; h < pl->H; ++h) {
                 if (pl->head_view[h] != v) continue;
                 int slot = -1;
@@ -245,7 +263,15 @@ int mate_plan_destroy(mate_plan_t *plan) {
 int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len,
               const uint8_t *head_view, int H, int max_row_id, int max_col_id, void *stream,
               mate_plan_t **out) {
+    return mate_plan_bucketed(row_ids, col_ids, B, N, prefix_len, head_view, H, max_row_id, max_col_id, 0,
+                              stream, out);
+}
+
+int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len,
+                       const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
+                       void *stream, mate_plan_t **out) {
     if (out) *out = nullptr;
+    if (radius < 0) return MATE_ERR_INVALID_ARG;
     if (!row_ids || !col_ids || !head_view || !out) return MATE_ERR_INVALID_ARG;
     if (B <= 0 || N <= 0 || H <= 0 || prefix_len < 0 || prefix_len > N) return MATE_ERR_INVALID_ARG;
     if (max_row_id < 0 || max_col_id < 0) return MATE_ERR_INVALID_ARG;
@@ -261,6 +287,7 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
     pl->N = N;
     pl->P = prefix_len;
     pl->H = H;
+    pl->radius = radius;
     pl->head_view.assign(head_view, head_view + H);
     pl->view[0].max_id = max_row_id;
     pl->view[1].max_id = max_col_id;
@@ -290,7 +317,7 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
     bool ok = cudaMemsetAsync(pl->status_dev, 0, 4 * sizeof(int32_t), st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(pl->head_view_dev, pl->head_view.data(), H, cudaMemcpyHostToDevice,
                                st) == cudaSuccess;
-    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, prefix_len, pl->view[0], pl->view[1],
+    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, prefix_len, radius, pl->view[0], pl->view[1],
                                          pl->n_valid_dev, pl->status_dev, st) == cudaSuccess;
     for (int v = 0; v < 2 && ok; ++v) {
         seg_off_host[v].resize((size_t)B * (pl->view[v].max_id + 2));
@@ -310,16 +337,22 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
         return rc;
     }
 
-    // unmasked pairs per (example, view): P * n_valid + sum_s L_s (L_s + P)
+    // unmasked pairs per (example, view): P * n_valid + sum_s L_s (L_s + P); a bucketed plan counts,
+    // row by row, the prefix and the clipped part of the segment
     pl->pairs.assign((size_t)B * 2, 0);
     for (int v = 0; v < 2; ++v) {
         const int S = pl->view[v].max_id + 2;
         for (int b = 0; b < B; ++b) {
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
             int64_t c = (int64_t)prefix_len * pl->n_valid[b];
-            for (int s = 0; s + 1 < S; ++s) {
-                const int64_t L = so[s + 1] - so[s];
-                c += L * (L + prefix_len);
+            if (radius > 0) {
+                const RowBounds rb{so, S, prefix_len, radius};
+                for (int t = prefix_len; t < pl->n_valid[b]; ++t) c += prefix_len + rb.hi(t) - rb.lo(t);
+            } else {
+                for (int s = 0; s + 1 < S; ++s) {
+                    const int64_t L = so[s + 1] - so[s];
+                    c += L * (L + prefix_len);
+                }
             }
             pl->pairs[(size_t)b * 2 + v] = c;
         }

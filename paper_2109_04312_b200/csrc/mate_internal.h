@@ -41,7 +41,8 @@ struct ViewPlan {
     int32_t *perm = nullptr;      // [B, N]   view position -> original position
     int32_t *inv_perm = nullptr;  // [B, N]
     int32_t *seg_off = nullptr;   // [B, max_id + 2]
-    int32_t *seg_lo = nullptr;    // [B, N]   per view position: first key of its own segment
+    int32_t *seg_lo = nullptr;    // [B, N]   per view position: first key of its own segment (bucketed
+                                  //          plans: of the part of it within the adjacent buckets)
     int32_t *seg_hi = nullptr;    // [B, N]   one past the last key (prefix rows: n_valid; padding: 0)
     int32_t *cursor = nullptr;    // [B, max_id + 2] scratch of the counting sort
     int max_id = 0;
@@ -52,6 +53,7 @@ struct ViewPlan {
 
 struct mate_plan_s {
     int B = 0, N = 0, P = 0, H = 0;
+    int radius = 0;                      // > 0: bucketed pattern (Section 3.1), buckets of this many positions
     std::vector<uint8_t> head_view;      // host copy
     uint8_t *head_view_dev = nullptr;    // [H]
     mate::ViewPlan view[2];
@@ -83,7 +85,7 @@ namespace mate {
 
 // plan kernels (mate_plan_kernels.cu)
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P,
-                                const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
+                                int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
                                 int32_t *status, cudaStream_t stream);
 
 // SIMT kernels (mate_simt.cu)

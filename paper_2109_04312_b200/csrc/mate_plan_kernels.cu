@@ -20,7 +20,7 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane) {
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N, int P,
+plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N, int P, int radius,
             ViewPlan rowv, ViewPlan colv, int32_t *__restrict__ n_valid_out,
             int32_t *__restrict__ status) {
     __shared__ int32_t s_cursor[kSmemIds];
@@ -119,7 +119,9 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
     }
     __syncthreads();
 
-    // 4. per view position: the key range of its own segment
+    // 4. per view position: the key range of its own segment.  With a radius (the bucketed form of
+    //    Section 3.1: the order behind the prefix is cut into buckets of `radius` positions and a
+    //    token sees its own bucket and the two next to it) the range is clipped to those buckets.
     int32_t *seg_lo = vp.seg_lo + (size_t)b * N, *seg_hi = vp.seg_hi + (size_t)b * N;
     for (int t = tid; t < N; t += kPlanThreads) {
         int lo = 0, hi = 0;
@@ -129,6 +131,12 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
             int id = ids[perm[t]];
             lo = seg_off[id];
             hi = seg_off[id + 1];
+            if (radius > 0) {
+                const long long bk = (t - P) / radius;
+                const long long w0 = P + (bk - 1) * radius, w1 = P + (bk + 2) * radius;
+                lo = (int)max((long long)lo, w0);
+                hi = (int)min((long long)hi, w1);
+            }
         }
         seg_lo[t] = lo;
         seg_hi[t] = hi;
@@ -138,10 +146,10 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
 }  // namespace
 
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P,
-                                const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
+                                int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
                                 int32_t *status, cudaStream_t stream) {
     dim3 grid(B, 2);
-    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, P, rowv, colv, n_valid,
+    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, P, radius, rowv, colv, n_valid,
                                                    status);
     return cudaGetLastError();
 }
