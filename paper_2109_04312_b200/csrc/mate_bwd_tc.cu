@@ -402,34 +402,47 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                         tc_wait_ld();
                         TR_ADD(4, t_ld);
                         if (cc == last_ld) signal_st();
+                        // Rounds that lie inside the segment of every row of the warp take the
+                        // path without the per-element column test (the side and this flag are
+                        // compile-time constants inside).  Two columns at a time, packed fp32.
                         const bool full = cb >= e_lo_max && cb + kRound <= e_hi_min;
+                        const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+                        const uint64_t row_nlse2 = pack_f32x2(-row_lse2, -row_lse2), row_D2 = pack_f32x2(row_D, row_D);
+                        auto math = [&](auto full_tag) {
+                            constexpr bool kFull = decltype(full_tag)::value;
 #pragma unroll
-                        for (int e = 0; e < kRound; e += 4) {
-                            float lse2[4], Dv[4];
-                            if (kKeySide) {
-                                const float4 a = vec4[(cb + e) >> 2], d4 = vec4[32 + ((cb + e) >> 2)];
-                                lse2[0] = a.x; lse2[1] = a.y; lse2[2] = a.z; lse2[3] = a.w;
-                                Dv[0] = d4.x; Dv[1] = d4.y; Dv[2] = d4.z; Dv[3] = d4.w;
-                            } else {
+                            for (int e = 0; e < kRound; e += 4) {
+                                uint64_t nlse[2], Dv[2];
+                                if (kKeySide) {
+                                    const float4 a = vec4[(cb + e) >> 2], d4 = vec4[32 + ((cb + e) >> 2)];
+                                    nlse[0] = pack_f32x2(a.x, a.y);  // the loaders store -LSE
+                                    nlse[1] = pack_f32x2(a.z, a.w);
+                                    Dv[0] = pack_f32x2(d4.x, d4.y);
+                                    Dv[1] = pack_f32x2(d4.z, d4.w);
+                                } else {
+                                    nlse[0] = nlse[1] = row_nlse2;
+                                    Dv[0] = Dv[1] = row_D2;
+                                }
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    lse2[q] = row_lse2;
-                                    Dv[q] = row_D;
+                                for (int q = 0; q < 2; ++q) {
+                                    const int k = e + 2 * q;
+                                    float x0, x1;
+                                    unpack_f32x2(fma_f32x2(pack_f32x2(sv[k], sv[k + 1]), scale2, nlse[q]), x0, x1);
+                                    float p0 = ex2(x0), p1 = ex2(x1);
+                                    if (!kFull) {
+                                        if ((uint32_t)(cb + k - r_lo) >= r_span) p0 = 0.f;
+                                        if ((uint32_t)(cb + k + 1 - r_lo) >= r_span) p1 = 0.f;
+                                    }
+                                    float d0, d1;
+                                    unpack_f32x2(mul_f32x2(pack_f32x2(p0, p1), sub_f32x2(pack_f32x2(tv[k], tv[k + 1]), Dv[q])),
+                                                 d0, d1);
+                                    pk_p[k >> 1] = pack_bf16(p0, p1);
+                                    pk_ds[k >> 1] = pack_bf16(d0, d1);
                                 }
                             }
-                            float pv[4], dsv[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const float xx = fmaf(__uint_as_float(sv[e + q]), p.scale_log2, -lse2[q]);
-                                pv[q] = ex2(xx);
-                                if (!full && (uint32_t)(cb + e + q - r_lo) >= r_span) pv[q] = 0.f;
-                                dsv[q] = pv[q] * (__uint_as_float(tv[e + q]) - Dv[q]);
-                            }
-                            pk_p[e >> 1] = pack_bf16(pv[0], pv[1]);
-                            pk_p[(e >> 1) + 1] = pack_bf16(pv[2], pv[3]);
-                            pk_ds[e >> 1] = pack_bf16(dsv[0], dsv[1]);
-                            pk_ds[(e >> 1) + 1] = pack_bf16(dsv[2], dsv[3]);
-                        }
+                        };
+                        if (full) math(std::true_type{});
+                        else math(std::false_type{});
                     }
                     if (!a_free) {
                         TR_T0(t_wg);
@@ -736,7 +749,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                         const int cidx = ltid + q * kLoadThreads;
                         if (cidx < kTile) {
                             const int o = perm[t.k0 + min(cidx, t.w - 1)];
-                            v_lse[q] = p.LSE[bh + o] * 1.4426950408889634f;
+                            v_lse[q] = p.LSE[bh + o] * -1.4426950408889634f;  // stored negated: the addend of the exponent
                             v_D[q] = p.D[bh + o];
                         }
                     }

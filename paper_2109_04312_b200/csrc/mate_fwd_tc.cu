@@ -169,45 +169,47 @@ __device__ __forceinline__ void copy_rows(uint32_t s_tile, const __nv_bfloat16 *
     }
 }
 
-// Row max over one chunk of 32 scores (tile-local columns cb .. cb + 31); a column c counts for the
-// row iff r_lo <= c < r_lo + r_span, and `full` says that every column of the chunk counts.
-__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], int cb, bool full, int r_lo,
-                                          uint32_t r_span, float (&tm)[4]) {
-    if (full) {
+// A chunk is 32 scores of one row (tile-local columns cb .. cb + 31).  A column c counts for the row
+// iff r_lo <= c < r_lo + r_span; the scores of the other columns are replaced by -inf, which the row
+// max ignores and the exponential turns into an exact 0 (the scale is positive).
+__device__ __forceinline__ void chunk_mask(uint32_t (&v)[32], int cb, int r_lo, uint32_t r_span) {
 #pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-            tm[0] = fmax3(tm[0], __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
-            tm[1] = fmax3(tm[1], __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-            tm[2] = fmax3(tm[2], __uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
-            tm[3] = fmax3(tm[3], __uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-        }
-    } else {
+    for (int e = 0; e < 32; ++e)
+        if ((uint32_t)(cb + e - r_lo) >= r_span) v[e] = 0xff800000u;
+}
+// Row max over one chunk, four partial maxima.
+__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], float (&tm)[4]) {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-            const bool ok = (uint32_t)(cb + e - r_lo) < r_span;
-            tm[e & 3] = fmaxf(tm[e & 3], ok ? __uint_as_float(v[e]) : -INFINITY);
-        }
+    for (int e = 0; e < 32; e += 8) {
+        tm[0] = fmax3(tm[0], __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+        tm[1] = fmax3(tm[1], __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+        tm[2] = fmax3(tm[2], __uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+        tm[3] = fmax3(tm[3], __uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
     }
 }
-// P of one chunk: exp2(s * scale_log2 + neg_m) for the columns that count, 0 elsewhere, packed as
-// bf16 pairs (even column in the low half); adds the row sums of even / odd columns to l0 / l1.
-__device__ __forceinline__ void chunk_exp(const uint32_t (&v)[32], int cb, bool full, int r_lo,
-                                          uint32_t r_span, float scale_log2, float neg_m,
-                                          uint32_t (&packed)[16], float &l0, float &l1) {
+// P of one chunk: exp2(s * scale_log2 + neg_m), packed as bf16 pairs (even column in the low half);
+// the row sums go to two packed pairs of partial sums.  The multiply-adds and the sums work on two
+// columns per instruction (packed fp32 pairs); only the exponential is per column.
+__device__ __forceinline__ void chunk_exp(const uint32_t (&v)[32], uint64_t scale2, uint64_t neg_m2,
+                                          uint32_t (&packed)[16], uint64_t &l01, uint64_t &l23) {
 #pragma unroll
-    for (int e = 0; e < 32; e += 2) {
-        float x0 = fmaf(__uint_as_float(v[e]), scale_log2, neg_m);
-        float x1 = fmaf(__uint_as_float(v[e + 1]), scale_log2, neg_m);
-        if (!full) {
-            if ((uint32_t)(cb + e - r_lo) >= r_span) x0 = -INFINITY;
-            if ((uint32_t)(cb + e + 1 - r_lo) >= r_span) x1 = -INFINITY;
-        }
-        const float p0 = ex2(x0), p1 = ex2(x1);
-        l0 += p0;
-        l1 += p1;
-        __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-        packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b2);
+    for (int e = 0; e < 32; e += 4) {
+        float x0, x1, x2, x3;
+        unpack_f32x2(fma_f32x2(pack_f32x2(v[e], v[e + 1]), scale2, neg_m2), x0, x1);
+        unpack_f32x2(fma_f32x2(pack_f32x2(v[e + 2], v[e + 3]), scale2, neg_m2), x2, x3);
+        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+        l01 = add_f32x2(l01, pack_f32x2(p0, p1));
+        l23 = add_f32x2(l23, pack_f32x2(p2, p3));
+        __nv_bfloat162 b01 = __floats2bfloat162_rn(p0, p1), b23 = __floats2bfloat162_rn(p2, p3);
+        packed[e >> 1] = *reinterpret_cast<uint32_t *>(&b01);
+        packed[(e >> 1) + 1] = *reinterpret_cast<uint32_t *>(&b23);
     }
+}
+__device__ __forceinline__ float sum_f32x2(uint64_t a, uint64_t b) {
+    float a0, a1, b0, b1;
+    unpack_f32x2(a, a0, a1);
+    unpack_f32x2(b, b0, b1);
+    return (a0 + a1) + (b0 + b1);
 }
 
 __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
@@ -396,7 +398,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     // one pass with the running max; the tile's own max is known before S is given up
                     float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                     const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
-                    float lsum = 0.f, lsum1 = 0.f;
+                    const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2), neg_m2 = pack_f32x2(neg_m, neg_m);
+                    uint64_t lsum = 0ull, lsum1 = 0ull;  // packed pairs of partial row sums
                     bool redo = false;
 #pragma unroll 1
                     for (int ch = ch0; ch < ch1; ++ch) {
@@ -409,15 +412,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                             uint32_t v[32];
                             tmem_ld32(tS + cb, v);
                             tc_wait_ld();
-                            const bool full = cb >= e_lo_max && cb + 32 <= e_hi_min;
-                            chunk_max(v, cb, full, r_lo, r_span, tm);
+                            if (!(cb >= e_lo_max && cb + 32 <= e_hi_min)) chunk_mask(v, cb, r_lo, r_span);
+                            chunk_max(v, tm);
                             if (ch == last_ld) {
                                 const float t2 = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
                                 redo = __any_sync(0xffffffffu, t2 > m2 + kRescaleThreshold);
                                 if (redo) break;
                                 release_s();
                             }
-                            chunk_exp(v, cb, full, r_lo, r_span, p.scale_log2, neg_m, packed, lsum, lsum1);
+                            chunk_exp(v, scale2, neg_m2, packed, lsum, lsum1);
                         }
                         if (!wait_pv()) break;
                         tmem_st16(tP + ch * 16, packed);
@@ -425,7 +428,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     if (!alive) break;
                     if (!redo) {
                         if (last_ld < 0) release_s();
-                        l += lsum + lsum1;
+                        l += sum_f32x2(lsum, lsum1);
                     }
                     two_pass = redo;
                 }
@@ -440,7 +443,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                         uint32_t v[32];
                         tmem_ld32(tS + cb, v);
                         tc_wait_ld();
-                        chunk_max(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, tm);
+                        if (!(cb >= e_lo_max && cb + 32 <= e_hi_min)) chunk_mask(v, cb, r_lo, r_span);
+                        chunk_max(v, tm);
                     }
                     const float tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
                     const float t2 = tmax * p.scale_log2;
@@ -467,7 +471,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                     const float neg_m = (m2 == -INFINITY) ? 0.f : -m2;
 
                     // pass 2: P = exp2(s * scale_log2 - m) as bf16 pairs into the P columns, row sum
-                    float lsum = 0.f, lsum1 = 0.f;
+                    const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2), neg_m2 = pack_f32x2(neg_m, neg_m);
+                    uint64_t lsum = 0ull, lsum1 = 0ull;
                     if (last_ld < 0) release_s();
 #pragma unroll 1
                     for (int ch = ch0; ch < ch1; ++ch) {
@@ -481,12 +486,12 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                             tmem_ld32(tS + cb, v);
                             tc_wait_ld();
                             if (ch == last_ld) release_s();
-                            chunk_exp(v, cb, cb >= e_lo_max && cb + 32 <= e_hi_min, r_lo, r_span, p.scale_log2, neg_m,
-                                      packed, lsum, lsum1);
+                            if (!(cb >= e_lo_max && cb + 32 <= e_hi_min)) chunk_mask(v, cb, r_lo, r_span);
+                            chunk_exp(v, scale2, neg_m2, packed, lsum, lsum1);
                         }
                         tmem_st16(tP + ch * 16, packed);
                     }
-                    l += lsum + lsum1;
+                    l += sum_f32x2(lsum, lsum1);
                 }
                 first = false;
 
