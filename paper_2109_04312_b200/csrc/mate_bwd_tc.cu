@@ -174,19 +174,30 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&b2);
 }
 
-// D_k = sum_e dO_ke O_ke per row (original order), one warp per row, d = 64.
+// D_k = sum_e dO_ke O_ke per row (original order), d = 64: eight threads per row, 16 bytes of each
+// tensor per thread.  The first thread also clears the work-item counter of the kernel that follows.
 __global__ void __launch_bounds__(256) rowdot_kernel(const __nv_bfloat16 *__restrict__ dO,
                                                      const __nv_bfloat16 *__restrict__ O,
-                                                     float *__restrict__ D, size_t rows) {
-    const size_t r = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (r >= rows) return;
-    const __nv_bfloat162 a = reinterpret_cast<const __nv_bfloat162 *>(dO + r * 64)[lane];
-    const __nv_bfloat162 b = reinterpret_cast<const __nv_bfloat162 *>(O + r * 64)[lane];
-    float acc = __bfloat162float(a.x) * __bfloat162float(b.x) + __bfloat162float(a.y) * __bfloat162float(b.y);
+                                                     float *__restrict__ D, size_t rows, int32_t *counter) {
+    if (blockIdx.x == 0 && threadIdx.x < 64) counter[threadIdx.x] = 0;
+    const size_t r = (size_t)blockIdx.x * 32 + (threadIdx.x >> 3);
+    const int part = threadIdx.x & 7;
+    float acc = 0.f;
+    if (r < rows) {
+        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(dO + r * 64) + part);
+        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(O + r * 64) + part);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) D[r] = acc;
+        for (int i = 0; i < 4; ++i) {
+            const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&aw[i]));
+            const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&bw[i]));
+            acc = fmaf(fa.x, fb.x, acc);
+            acc = fmaf(fa.y, fb.y, acc);
+        }
+    }
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (part == 0 && r < rows) D[r] = acc;
 }
 
 // Everything an item needs that does not depend on the role of the warp.
@@ -835,8 +846,8 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = plan->status_dev;
 
-    if (cudaMemsetAsync(ws, 0, 256, stream) != cudaSuccess) return MATE_ERR_CUDA;
-    rowdot_kernel<<<(unsigned)((bhn + 7) / 8), 256, 0, stream>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, D, bhn);
+    rowdot_kernel<<<(unsigned)((bhn + 31) / 32), 256, 0, stream>>>((const __nv_bfloat16 *)dO, (const __nv_bfloat16 *)O, D, bhn,
+                                                                   reinterpret_cast<int32_t *>(ws));
     tc_bwd_kernel<<<plan->n_ctas, kThreads, kSmemBytes, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
