@@ -753,16 +753,25 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
                 if (lane == 0) mbar_arrive(oldest);
             }
         };
-        // Signals every group still pending.  Called before this warp blocks on a buffer that is
-        // not free yet: the consumers may need exactly those groups to free it.
+        // Signals every group still pending, oldest first and each as soon as its own copies have
+        // landed (an older group is not held back by the latency of a newer one).  Called before
+        // this warp blocks on a buffer that is not free yet: the consumers may need exactly those
+        // groups to free it.
         auto flush = [&]() {
-            cp_async_wait_group<0>();
-            fence_proxy_async();
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < kLag; ++i) {
-                if (pend[i] && lane == 0) mbar_arrive(pend[i]);
-                pend[i] = 0;
+            static_assert(kLag == 2, "written out for two pending groups");
+            if (pend[0]) {
+                cp_async_wait_group<1>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pend[0]);
+                pend[0] = 0;
+            }
+            if (pend[1]) {
+                cp_async_wait_group<0>();
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pend[1]);
+                pend[1] = 0;
             }
         };
         auto wait_free = [&](uint32_t bar, uint32_t parity) -> bool {
