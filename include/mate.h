@@ -96,11 +96,21 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
                        const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
                        void *stream, mate_plan_t **out);
 
+/* The same with one prefix length per example (the paper's inputs are a question or a passage of
+ * varying length followed by the table, Section 3 and Section 5; its formula takes the set Q per
+ * example).  prefix_len is a HOST int32 [B] array, 0 <= prefix_len[b] <= N; examples of different
+ * total length are padded at the tail with negative ids as for mate_plan.  radius as for
+ * mate_plan_bucketed (0 = the exact pattern).  mate_plan and mate_plan_bucketed are this call with
+ * B equal entries.  All other arguments, ownership and errors as for mate_plan. */
+int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
+                     const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
+                     void *stream, mate_plan_t **out);
+
 /* Copies one view's order to HOST arrays (any pointer may be null to skip it):
  *   perm      int32 [B, N]          perm[b][t] = original position of the t-th token of the view
  *   inv_perm  int32 [B, N]          inverse of perm
  *   seg_off   int32 [B, max_id+2]   tokens with id s occupy view positions [seg_off[s], seg_off[s+1]);
- *                                   seg_off[0] = prefix_len, seg_off[max_id+1] = number of
+ *                                   seg_off[0] = prefix_len (of the example), seg_off[max_id+1] = number of
  *                                   non-padding tokens */
 int mate_plan_get(const mate_plan_t *plan, int view, int32_t *perm, int32_t *inv_perm,
                   int32_t *seg_off);

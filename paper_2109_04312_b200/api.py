@@ -42,6 +42,8 @@ def _load():
     lib.mate_plan.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_bucketed.restype = i32
     lib.mate_plan_bucketed.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
+    lib.mate_plan_varlen.restype = i32
+    lib.mate_plan_varlen.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_get.restype = i32
     lib.mate_plan_get.argtypes = [vp, i32, vp, vp, vp]
     lib.mate_plan_useful_pairs.restype = i32
@@ -136,8 +138,15 @@ def mate_plan_bucketed(row_ids, col_ids, prefix_len, head_view, radius, max_row_
     return mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id, max_col_id, radius=radius)
 
 
+def mate_plan_varlen(row_ids, col_ids, prefix_lens, head_view, radius=0, max_row_id=None, max_col_id=None) -> Plan:
+    """Plan with one prefix length per example (see mate_plan_varlen in mate.h): prefix_lens has B entries."""
+    return mate_plan(row_ids, col_ids, [int(x) for x in prefix_lens], head_view, max_row_id, max_col_id,
+                     radius=radius)
+
+
 def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_id=None, radius=0) -> Plan:
-    """row_ids, col_ids: int32 CUDA tensors [B, N]; head_view: sequence of 0 (row) / 1 (column)."""
+    """row_ids, col_ids: int32 CUDA tensors [B, N]; head_view: sequence of 0 (row) / 1 (column);
+    prefix_len: one int, or a list of B ints (one per example)."""
     if row_ids.dtype != torch.int32 or col_ids.dtype != torch.int32 or row_ids.shape != col_ids.shape \
             or row_ids.dim() != 2:
         raise ValueError("row_ids / col_ids must be int32 tensors of the same [B, N] shape")
@@ -150,17 +159,21 @@ def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_
     handle = C.c_void_p()
     with torch.cuda.device(row_ids.device):
         lib = _load()
-        if radius:
-            _check(lib.mate_plan_bucketed(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N,
-                                          int(prefix_len), hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
-                                          int(max_col_id), int(radius), _stream(), C.byref(handle)),
-                   "mate_plan_bucketed")
+        common = (_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N)
+        tail = (hv.ctypes.data, int(hv.shape[0]), int(max_row_id), int(max_col_id))
+        if isinstance(prefix_len, (list, tuple, np.ndarray)):
+            pf = np.ascontiguousarray(np.asarray(prefix_len, dtype=np.int32))
+            if pf.shape != (B,):
+                raise ValueError("prefix_len must have one entry per example")
+            _check(lib.mate_plan_varlen(*common, pf.ctypes.data, *tail, int(radius), _stream(), C.byref(handle)),
+                   "mate_plan_varlen")
+            prefix_len = pf.tolist()
+        elif radius:
+            _check(lib.mate_plan_bucketed(*common, int(prefix_len), *tail, int(radius), _stream(),
+                                          C.byref(handle)), "mate_plan_bucketed")
         else:
-            _check(lib.mate_plan(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N,
-                                 int(prefix_len), hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
-                                 int(max_col_id), _stream(), C.byref(handle)), "mate_plan")
-    return Plan(handle, B, N, int(prefix_len), int(hv.shape[0]), int(max_row_id), int(max_col_id),
-                row_ids.device)
+            _check(lib.mate_plan(*common, int(prefix_len), *tail, _stream(), C.byref(handle)), "mate_plan")
+    return Plan(handle, B, N, prefix_len, int(hv.shape[0]), int(max_row_id), int(max_col_id), row_ids.device)
 
 
 def mate_attn_workspace_bytes(plan, d, dtype, impl=IMPL_AUTO):

@@ -44,6 +44,7 @@ void carve(mate_plan_t *pl, char *base, size_t *total) {
         vp.cursor = c.take<int32_t>(S);
     }
     pl->n_valid_dev = c.take<int32_t>(pl->B);
+    pl->prefix_dev = c.take<int32_t>(pl->B);
     pl->status_dev = c.take<int32_t>(4);
     pl->head_view_dev = c.take<uint8_t>(pl->H);
     *total = align_up(c.off, 256);
@@ -106,7 +107,7 @@ int64_t half_cost(const FwdUnit &u, int h, const RowBounds &rb) {
 // shares is cut along the columns into parts of about 0.75 shares, to be combined in the kernel.
 void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_off_host, int64_t share,
                 std::vector<UnitCost> &all, int *n_slots, size_t *ws_bytes, int64_t *total_cost) {
-    const int P = pl->P, N = pl->N;
+    const int N = pl->N;
     all.clear();
     *n_slots = 0;
     *ws_bytes = 0;
@@ -118,6 +119,7 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
         for (int b = 0; b < pl->B; ++b) {
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
             const int nv = pl->n_valid[b];
+            const int P = pl->prefix[b];
             const RowBounds rb{so, S, P, pl->radius};
             std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
             for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
@@ -271,9 +273,21 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
                        const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
                        void *stream, mate_plan_t **out) {
     if (out) *out = nullptr;
+    if (B <= 0) return MATE_ERR_INVALID_ARG;
+    const std::vector<int32_t> prefix((size_t)B, prefix_len);
+    return mate_plan_varlen(row_ids, col_ids, B, N, prefix.data(), head_view, H, max_row_id, max_col_id, radius,
+                            stream, out);
+}
+
+int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
+                     const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
+                     void *stream, mate_plan_t **out) {
+    if (out) *out = nullptr;
     if (radius < 0) return MATE_ERR_INVALID_ARG;
-    if (!row_ids || !col_ids || !head_view || !out) return MATE_ERR_INVALID_ARG;
-    if (B <= 0 || N <= 0 || H <= 0 || prefix_len < 0 || prefix_len > N) return MATE_ERR_INVALID_ARG;
+    if (!row_ids || !col_ids || !head_view || !out || !prefix_len) return MATE_ERR_INVALID_ARG;
+    if (B <= 0 || N <= 0 || H <= 0) return MATE_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b)
+        if (prefix_len[b] < 0 || prefix_len[b] > N) return MATE_ERR_INVALID_ARG;
     if (max_row_id < 0 || max_col_id < 0) return MATE_ERR_INVALID_ARG;
     if ((long long)B * N > (1ll << 30) || max_row_id > (1 << 28) || max_col_id > (1 << 28))
         return MATE_ERR_UNSUPPORTED;
@@ -285,7 +299,7 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
     if (!pl) return MATE_ERR_NOMEM;
     pl->B = B;
     pl->N = N;
-    pl->P = prefix_len;
+    pl->prefix.assign(prefix_len, prefix_len + B);
     pl->H = H;
     pl->radius = radius;
     pl->head_view.assign(head_view, head_view + H);
@@ -317,7 +331,9 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
     bool ok = cudaMemsetAsync(pl->status_dev, 0, 4 * sizeof(int32_t), st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(pl->head_view_dev, pl->head_view.data(), H, cudaMemcpyHostToDevice,
                                st) == cudaSuccess;
-    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, prefix_len, radius, pl->view[0], pl->view[1],
+    ok = ok && cudaMemcpyAsync(pl->prefix_dev, pl->prefix.data(), B * sizeof(int32_t), cudaMemcpyHostToDevice,
+                               st) == cudaSuccess;
+    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, pl->prefix_dev, radius, pl->view[0], pl->view[1],
                                          pl->n_valid_dev, pl->status_dev, st) == cudaSuccess;
     for (int v = 0; v < 2 && ok; ++v) {
         seg_off_host[v].resize((size_t)B * (pl->view[v].max_id + 2));
@@ -344,14 +360,15 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
         const int S = pl->view[v].max_id + 2;
         for (int b = 0; b < B; ++b) {
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
-            int64_t c = (int64_t)prefix_len * pl->n_valid[b];
+            const int P = pl->prefix[b];
+            int64_t c = (int64_t)P * pl->n_valid[b];
             if (radius > 0) {
-                const RowBounds rb{so, S, prefix_len, radius};
-                for (int t = prefix_len; t < pl->n_valid[b]; ++t) c += prefix_len + rb.hi(t) - rb.lo(t);
+                const RowBounds rb{so, S, P, radius};
+                for (int t = P; t < pl->n_valid[b]; ++t) c += P + rb.hi(t) - rb.lo(t);
             } else {
                 for (int s = 0; s + 1 < S; ++s) {
                     const int64_t L = so[s + 1] - so[s];
-                    c += L * (L + prefix_len);
+                    c += L * (L + P);
                 }
             }
             pl->pairs[(size_t)b * 2 + v] = c;

@@ -87,7 +87,7 @@ struct Params {
     ViewPlan rowv, colv;
     const uint8_t *head_view;
     const FwdUnit *units;
-    int n_units, N, H, P;
+    int n_units, N, H;
     float scale, scale_log2;
     int32_t *status;
     int32_t *counter;      // next work item (zeroed before the launch)
@@ -850,7 +850,6 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.n_units = plan->n_bwd_units;
     p.N = plan->N;
     p.H = plan->H;
-    p.P = plan->P;
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = plan->status_dev;

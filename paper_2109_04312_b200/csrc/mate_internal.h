@@ -52,7 +52,9 @@ struct ViewPlan {
 }  // namespace mate
 
 struct mate_plan_s {
-    int B = 0, N = 0, P = 0, H = 0;
+    int B = 0, N = 0, H = 0;
+    std::vector<int32_t> prefix;         // |Q| per example (host copy)
+    int32_t *prefix_dev = nullptr;       // [B]
     int radius = 0;                      // > 0: bucketed pattern (Section 3.1), buckets of this many positions
     std::vector<uint8_t> head_view;      // host copy
     uint8_t *head_view_dev = nullptr;    // [H]
@@ -84,8 +86,8 @@ struct mate_plan_s {
 namespace mate {
 
 // plan kernels (mate_plan_kernels.cu)
-cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P,
-                                int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
+cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,
+                                const int32_t *prefix /* device [B] */, int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
                                 int32_t *status, cudaStream_t stream);
 
 // SIMT kernels (mate_simt.cu)

@@ -20,13 +20,15 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane) {
 }
 
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N, int P, int radius,
+plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N,
+            const int32_t *__restrict__ prefix, int radius,
             ViewPlan rowv, ViewPlan colv, int32_t *__restrict__ n_valid_out,
             int32_t *__restrict__ status) {
     __shared__ int32_t s_cursor[kSmemIds];
     __shared__ int s_n_valid;
 
     const int b = blockIdx.x, view = blockIdx.y;
+    const int P = prefix[b];  // |Q| of this example
     const ViewPlan &vp = view ? colv : rowv;
     const int32_t *ids = (view ? col_ids : row_ids) + (size_t)b * N;
     const int32_t *oth = (view ? row_ids : col_ids) + (size_t)b * N;
@@ -145,11 +147,11 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
 
 }  // namespace
 
-cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P,
-                                int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
+cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,
+                                const int32_t *prefix, int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
                                 int32_t *status, cudaStream_t stream) {
     dim3 grid(B, 2);
-    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, P, radius, rowv, colv, n_valid,
+    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, prefix, radius, rowv, colv, n_valid,
                                                    status);
     return cudaGetLastError();
 }

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__restrict__ V,
                 T *__restrict__ O, float *__restrict__ LSE, ViewPlan rowv, ViewPlan colv,
                 const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
-                int P, int d, float scale) {
+                const int32_t *__restrict__ prefix, int d, float scale) {
     __shared__ float s_q[kWarpsPerBlock][kMaxD];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kWarpsPerBlock + warp;
@@ -97,6 +97,7 @@ simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
 #pragma unroll
     for (int i = 0; i < kAccPerLane; ++i) acc[i] = 0.f;
 
+    const int P = prefix[b];
     const int lo = max(c.seg_lo[t], P), hi = c.seg_hi[t];
     for (int range = 0; range < 2; ++range) {
         const int j_begin = range ? lo : 0, j_end = range ? hi : P;
@@ -159,7 +160,7 @@ simt_bwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
                 const float *__restrict__ D, T *__restrict__ dQ, T *__restrict__ dK,
                 T *__restrict__ dV, ViewPlan rowv, ViewPlan colv,
                 const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
-                int P, int d, float scale) {
+                const int32_t *__restrict__ prefix, int d, float scale) {
     __shared__ float s_a[kWarpsPerBlock][kMaxD];  // own q (dQ) or own k (dK/dV)
     __shared__ float s_b[kWarpsPerBlock][kMaxD];  // own dO (dQ) or own v (dK/dV)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -194,6 +195,7 @@ simt_bwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
 #pragma unroll
     for (int i = 0; i < kAccPerLane; ++i) acc0[i] = acc1[i] = 0.f;
 
+    const int P = prefix[b];
     const int lo = max(c.seg_lo[t], P), hi = c.seg_hi[t];
     for (int range = 0; range < 2; ++range) {
         const int j_begin = range ? lo : 0, j_end = range ? hi : P;
@@ -248,7 +250,7 @@ int simt_fwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *
     dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
     simt_fwd_kernel<T><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (T *)O, LSE, pl->view[0], pl->view[1],
-        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->P, d, scale);
+        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->prefix_dev, d, scale);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
@@ -263,10 +265,10 @@ int simt_bwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *
     dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
     simt_bwd_kernel<T, false><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
-        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->P, d, scale);
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->prefix_dev, d, scale);
     simt_bwd_kernel<T, true><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
-        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->P, d, scale);
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->prefix_dev, d, scale);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
