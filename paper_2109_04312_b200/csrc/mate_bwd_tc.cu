@@ -276,6 +276,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
 #endif
     // every wait is bounded; the first one to expire raises the abort flag, which ends all roles
     auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+        if (mbar_test_wait(bar, parity)) return true;  // already complete: no trip through the suspending form
         for (uint32_t it = 0; it < kWaitLimit; ++it) {
             if (mbar_try_wait(bar, parity)) return true;
             if (*s_abort) return false;
