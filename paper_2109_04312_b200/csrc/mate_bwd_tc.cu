@@ -469,7 +469,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
                 }
                 if (!alive) break;
                 if (!st_signalled) signal_st();
-                if (!a_free) {  // nothing written in this tile: the phase is consumed all the same
+                // Nothing written in this tile: the phase is consumed all the same.  The wait also keeps this
+                // warp's arrival below out of the barrier phase of the previous tile, which a slower
+                // warp may not have reached yet (two arrivals of one warp would complete it early).
+                if (!a_free) {
                     if (!(alive = wait(bars + 8 * kBarGDone, ph_g))) break;
                     ph_g ^= 1;
                 }
