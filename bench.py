@@ -29,7 +29,7 @@ UNIT = "TFLOP/s"
 N_BUFFER_SETS = 4
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (same workload; None until a capture exists)
-NCU_TRAFFIC_BYTES = {"tc_fwd_kernel": 34.32e6 + 0.15e6, "tc_bwd_kernel": 47.42e6 + 6.82e6}
+NCU_TRAFFIC_BYTES = {"tc_fwd_kernel": 34.32e6 + 0.29e6, "tc_bwd_kernel": 47.46e6 + 6.33e6}
 
 
 def load_peaks():
