@@ -98,7 +98,7 @@ def test_bucketed_plan_counts_the_oracles_pairs(name, R):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("name,R", [("bert", 42), ("bert", 5), ("medium", 42), ("medium", 7), ("skew", 42)])
+@pytest.mark.parametrize("name,R", [("bert", 42), ("bert", 5), ("bert", 1), ("medium", 42), ("medium", 7), ("skew", 42)])
 @pytest.mark.parametrize("impl_idx", [0, 1], ids=["simt", "tc"])
 def test_bucketed_forward_backward_parity(name, R, impl_idx):
     import torch

@@ -117,3 +117,43 @@ def test_varlen_forward_backward_parity(impl_idx, radius):
         for nm, g, o in zip(("dQ", "dK", "dV"), grads, og):
             hp.assert_close(g[sl], o, atol, rtol, "%s of example %d" % (nm, b))
     plan.destroy()
+
+
+@pytest.mark.parametrize("impl_idx", [0, 1], ids=["simt", "tc"])
+def test_varlen_degenerate_examples(impl_idx):
+    """A batch whose examples are: only padding, only a prefix that fills the sequence, no prefix at
+    all, and a prefix followed by padding only."""
+    import torch
+    N, H, d = 300, 2, 64
+    r0 = np.full((1, N), -1, np.int32)
+    r1 = np.zeros((1, N), np.int32)
+    r2, c2 = tables.custom_structure(0, [(r, c, 2) for r in range(1, 11) for c in range(1, 8)], N)
+    r3 = np.full((1, N), -1, np.int32)
+    r3[0, :17] = 0
+    rows = np.concatenate([r0, r1, r2, r3])
+    cols = np.concatenate([r0, r1, c2, r3])
+    prefix = [0, N, 0, 17]
+    cfg = tables.TableConfig("degenerate", 4, H, 1, d, N, 0, 0, 0, "uniform", 1, 1, "bf16", 0.5)
+    vals = tables.make_values(cfg, N, 11)
+    hv = tables.head_view(cfg)
+    m, plan = make_plan(rows, cols, prefix, hv)
+    impl = (m.IMPL_SIMT, m.IMPL_TCGEN05)[impl_idx]
+    scale = 0.125
+    atol, rtol = hp.tol("bf16")
+    Q, K, V, dO = (hp.to_dev(vals[n], "bf16") for n in ("Q", "K", "V", "dO"))
+    O, LSE = m.mate_attn_fwd(plan, Q, K, V, scale, impl)
+    dQ, dK, dV = m.mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale, impl)
+    torch.cuda.synchronize()
+    plan.status()
+    gO, grads = hp.to_np(O), [hp.to_np(g) for g in (dQ, dK, dV)]
+    for b, P in enumerate(prefix):
+        sl = slice(b, b + 1)
+        ex = {n: vals[n][sl] for n in vals}
+        oO, _ = oracle.fwd(ex["Q"], ex["K"], ex["V"], rows[sl], cols[sl], P, hv, scale)
+        og = oracle.bwd(ex["Q"], ex["K"], ex["V"], ex["dO"], rows[sl], cols[sl], P, hv, scale)
+        hp.assert_close(gO[sl], oO, atol, rtol, "O of example %d" % b)
+        for nm, g, o in zip(("dQ", "dK", "dV"), grads, og):
+            hp.assert_close(g[sl], o, atol, rtol, "%s of example %d" % (nm, b))
+    assert np.all(gO[0] == 0) and all(np.all(g[0] == 0) for g in grads)  # the all-padding example
+    plan.destroy()
+
