@@ -74,9 +74,15 @@ const char *mate_status_string(int status);
  *   max_row_id, max_col_id   inclusive upper bounds of the non-negative ids
  *   out               receives a plan owned by the library; free it with mate_plan_destroy
  *
- * The plan can be reused for any number of forward/backward calls, layers and head dims.  Runs its
- * kernels on `stream` and waits for them (it allocates device memory, so call it outside a stream
- * capture).  Ids that break the conventions give MATE_ERR_INVALID_ARG and no plan. */
+ * The plan can be reused for any number of forward/backward calls, layers and head dims, on the
+ * device that was current when it was made (calls with another device current return
+ * MATE_ERR_INVALID_ARG).  It also holds a few scheduling counters of the tensor-core forward, so
+ * calls that use ONE plan -- mate_attn_fwd, mate_plan_status -- must not overlap on the GPU: put
+ * them on one stream or order them with events.  Work that should overlap (two streams) needs one
+ * plan per stream; mate_attn_bwd keeps its counters in its workspace and only needs separate
+ * workspaces.  Runs its kernels on `stream` and waits for them (it allocates device memory, so call
+ * it outside a stream capture).  Ids that break the conventions give MATE_ERR_INVALID_ARG and no
+ * plan. */
 int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len,
               const uint8_t *head_view, int H, int max_row_id, int max_col_id, void *stream,
               mate_plan_t **out);
@@ -136,7 +142,10 @@ int mate_attn_workspace_bytes(const mate_plan_t *plan, int d, int dtype, unsigne
  *   O         [B, H, N, d] same type, fully overwritten, original token order
  *   LSE       float32 [B, H, N]
  *   workspace device scratch of at least fwd_bytes (may be null when that is 0), 256-byte aligned;
- *             contents are undefined afterwards; concurrent calls need separate workspaces
+ *             contents are undefined afterwards; concurrent calls need separate workspaces AND
+ *             separate plans (see mate_plan)
+ *   scale     any finite value.  The tensor-core kernels need scale > 0; with MATE_IMPL_AUTO other
+ *             values run on the SIMT kernels, with MATE_IMPL_TCGEN05 they give MATE_ERR_UNSUPPORTED
  * d must be a multiple of 8 and at most 128.  Asynchronous on `stream`. */
 int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d,
                   int dtype, float scale, void *O, float *LSE, void *workspace,

@@ -314,6 +314,7 @@ int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int 
             delete pl;
             return MATE_ERR_CUDA;
         }
+        pl->device = dev;
     }
     size_t total = 0;
     carve(pl, nullptr, &total);
@@ -438,6 +439,14 @@ int mate_plan_status(const mate_plan_t *plan, void *stream) {
     return MATE_OK;
 }
 
+// The plan's arrays, its CTA count and the kernels' per-device set-up belong to the device the plan
+// was made on: a call with another device current is refused before anything is launched.
+static int check_device(const mate_plan_t *plan) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MATE_ERR_CUDA;
+    return dev == plan->device ? MATE_OK : MATE_ERR_INVALID_ARG;
+}
+
 static int check_common(const mate_plan_t *plan, int d, int dtype, unsigned flags, bool *use_tc) {
     if (!plan) return MATE_ERR_INVALID_ARG;
     if (dtype != MATE_BF16 && dtype != MATE_F32) return MATE_ERR_UNSUPPORTED;
@@ -466,10 +475,16 @@ int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     bool use_tc = false;
     int rc = check_common(plan, d, dtype, flags, &use_tc);
     if (rc != MATE_OK) return rc;
+    if ((rc = check_device(plan)) != MATE_OK) return rc;
     if (!Q || !K || !V || !O || !LSE) return MATE_ERR_INVALID_ARG;
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(LSE))
         return MATE_ERR_ALIGNMENT;
     cudaStream_t st = (cudaStream_t)stream;
+    // the tensor-core forward takes the row maximum before scaling, which needs scale > 0
+    if (use_tc && !(scale > 0.f)) {
+        if ((flags & 3u) == MATE_IMPL_TCGEN05) return MATE_ERR_UNSUPPORTED;
+        use_tc = false;
+    }
     if (use_tc) {
         const size_t need = mate::tc_fwd_workspace(plan, d);
         if (need > 0 && (!workspace || workspace_bytes < need)) return MATE_ERR_WORKSPACE;
@@ -486,6 +501,7 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     bool use_tc = false;
     int rc = check_common(plan, d, dtype, flags, &use_tc);
     if (rc != MATE_OK) return rc;
+    if ((rc = check_device(plan)) != MATE_OK) return rc;
     if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return MATE_ERR_INVALID_ARG;
     const void *ptrs[] = {Q, K, V, O, LSE, dO, dQ, dK, dV};
     for (const void *p : ptrs)

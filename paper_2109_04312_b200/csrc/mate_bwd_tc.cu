@@ -812,7 +812,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
     if (warp == kMmaWarp) tmem_dealloc(tmem, 512);
 }
 
-bool g_attr_set = false;
+SmemAttrOnce g_smem_attr;
 
 inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
@@ -827,12 +827,7 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
            const float *LSE, const void *dO, float scale, void *dQ, void *dK, void *dV, void *workspace,
            cudaStream_t stream) {
     if (plan->n_bwd_units == 0) return MATE_OK;
-    if (!g_attr_set) {
-        if (cudaFuncSetAttribute(tc_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSmemBytes) != cudaSuccess)
-            return MATE_ERR_CUDA;
-        g_attr_set = true;
-    }
+    if (g_smem_attr.ensure((const void *)tc_bwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
     const size_t bhn = (size_t)plan->B * plan->H * plan->N;
     uint8_t *ws = (uint8_t *)workspace;
     Params p;

@@ -895,7 +895,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     }
 }
 
-bool g_attr_set = false;
+SmemAttrOnce g_smem_attr;
 
 }  // namespace
 
@@ -907,12 +907,7 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
            float *LSE, void *workspace, cudaStream_t stream) {
     if (!(scale > 0.f)) return MATE_ERR_UNSUPPORTED;  // the row max is taken before scaling
     if (plan->n_fwd_units == 0) return MATE_OK;
-    if (!g_attr_set) {
-        if (cudaFuncSetAttribute(tc_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSmemBytes) != cudaSuccess)
-            return MATE_ERR_CUDA;
-        g_attr_set = true;
-    }
+    if (g_smem_attr.ensure((const void *)tc_fwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
     Params p;
     p.Q = (const __nv_bfloat16 *)Q;
     p.K = (const __nv_bfloat16 *)K;

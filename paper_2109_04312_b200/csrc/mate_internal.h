@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
 #include <vector>
 
 #include "mate.h"
@@ -53,6 +54,7 @@ struct ViewPlan {
 
 struct mate_plan_s {
     int B = 0, N = 0, H = 0;
+    int device = 0;                      // ordinal of the device the plan's arrays live on
     std::vector<int32_t> prefix;         // |Q| per example (host copy)
     int32_t *prefix_dev = nullptr;       // [B]
     int radius = 0;                      // > 0: bucketed pattern (Section 3.1), buckets of this many positions
@@ -84,6 +86,24 @@ struct mate_plan_s {
 };
 
 namespace mate {
+
+// Raises a kernel's dynamic shared-memory limit once per device.  cudaFuncSetAttribute acts on the
+// device that is current when it is called, so the "already done" flags are kept per device ordinal
+// (under a mutex: host threads may drive different devices at the same time).
+struct SmemAttrOnce {
+    static constexpr int kMaxDevices = 64;
+    std::mutex mu;
+    bool done[kMaxDevices] = {};
+    // returns MATE_OK or MATE_ERR_CUDA; `device` is the current device
+    int ensure(const void *kernel, int bytes, int device) {
+        std::lock_guard<std::mutex> lock(mu);
+        if (device >= 0 && device < kMaxDevices && done[device]) return MATE_OK;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+            return MATE_ERR_CUDA;
+        if (device >= 0 && device < kMaxDevices) done[device] = true;
+        return MATE_OK;
+    }
+};
 
 // plan kernels (mate_plan_kernels.cu)
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,

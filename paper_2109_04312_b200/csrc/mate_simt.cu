@@ -320,6 +320,7 @@ extern "C" int mate_attn_bwd_noalloc(const mate_plan_t *plan, const void *Q, con
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return MATE_ERR_CUDA;
     if (dev < 0 || dev >= kMaxDevices) return MATE_ERR_UNSUPPORTED;
+    if (dev != plan->device) return MATE_ERR_INVALID_ARG;  // the plan's arrays live on another device
     float *scratch = nullptr;
     {
         std::lock_guard<std::mutex> lock(mu);

@@ -102,7 +102,12 @@ def test_plan_rejects_bad_ids():
 
 # -------------------------------------------------------------------------------- forward / backward
 
-def run_case(cfg, rows, cols, vals, impl, head_view=None, backward=None, scale=None):
+def run_case(cfg, rows, cols, vals, impl, head_view=None, backward=None, scale=None, unit_grads=False):
+    """Forward (and backward) through the C ABI against the oracle.  unit_grads: for inputs much
+    larger than the usual N(0,1)/2 -- whose gradients would be tens of times larger too, while the
+    tolerance has a fixed absolute part -- dO is multiplied by a power of two chosen so that dQ keeps
+    its usual size (root mean square about 1/4).  The backward is linear in dO and a power of two is
+    exact, so the oracle's gradients are scaled by the same factor."""
     m = mate()
     plan, hv = make_plan(cfg, rows, cols, head_view)
     scale = (1.0 / np.sqrt(cfg.d)) if scale is None else scale
@@ -121,10 +126,15 @@ def run_case(cfg, rows, cols, vals, impl, head_view=None, backward=None, scale=N
     hp.assert_close(gLSE[vmask], oLSE[vmask], atol, rtol, "LSE")
     do_bwd = cfg.backward if backward is None else backward
     if do_bwd:
+        odQ, odK, odV = oracle.bwd(vals["Q"], vals["K"], vals["V"], vals["dO"], rows, cols, cfg.P, hv, scale)
+        if unit_grads:
+            rms = float(np.sqrt(np.mean(np.square(odQ[np.broadcast_to(valid[:, None, :, None], odQ.shape)]))))
+            f = 2.0 ** min(0, int(np.floor(np.log2(0.25 / max(rms, 1e-30)))))
+            dO = (dO.float() * f).to(dO.dtype)
+            odQ, odK, odV = odQ * f, odK * f, odV * f
         dQ, dK, dV = m.mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale, impl)
         torch.cuda.synchronize()
         plan.status()
-        odQ, odK, odV = oracle.bwd(vals["Q"], vals["K"], vals["V"], vals["dO"], rows, cols, cfg.P, hv, scale)
         for nm, g, o in (("dQ", dQ, odQ), ("dK", dK, odK), ("dV", dV, odV)):
             g = hp.to_np(g)
             hp.assert_close(g, o, atol, rtol, nm)
@@ -141,8 +151,10 @@ def test_tiny_fp32(seed):
 
 @pytest.mark.parametrize("name", ["bert", "medium", "long", "skew"])
 @pytest.mark.parametrize("impl_idx", [0, 1], ids=["simt", "tc"])
-def test_config_parity(name, impl_idx):
-    cfg, rows, cols, info, vals = hp.make_case(name)
+@pytest.mark.parametrize("seed", [1234, 21, 22])
+def test_config_parity(name, impl_idx, seed):
+    # three table structures (and value draws) per configuration; seed 1234 is the benchmark's
+    cfg, rows, cols, info, vals = hp.make_case(name, seed_structure=seed, seed_values=seed + 4444)
     run_case(cfg, rows, cols, vals, impls_for(cfg)[impl_idx])
 
 

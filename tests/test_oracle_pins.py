@@ -307,6 +307,26 @@ def test_bwd_against_autograd_of_masked_softmax():
     np.testing.assert_allclose(dV.sum(axis=2), dO[:, :, valid].sum(axis=2), rtol=1e-11)
 
 
+def test_batched_calls_equal_per_example_calls():
+    # The examples of a batch are independent (Section 3 defines the pattern per example): a call on
+    # B = 3 examples with different structures must return, example by example, what three B = 1
+    # calls return.  Pins the per-example offsets of every array inside the oracle's loops.
+    rows, cols, N = small_table(51, P=3, n_rows=3, n_cols=2, max_len=3, pad=2, B=3)
+    P, H, d, scale = 3, 3, 4, 0.8
+    hv = np.asarray([0, 1, 0], np.uint8)
+    Q, K, V, dO = rand_qkv(51, 3, H, N, d, k=4)
+    assert not np.array_equal(rows[0], rows[1]) and not np.array_equal(rows[1], rows[2])
+    O, LSE = oracle.fwd(Q, K, V, rows, cols, P, hv, scale)
+    dQ, dK, dV = oracle.bwd(Q, K, V, dO, rows, cols, P, hv, scale)
+    for b in range(3):
+        s = slice(b, b + 1)
+        O1, LSE1 = oracle.fwd(Q[s], K[s], V[s], rows[s], cols[s], P, hv, scale)
+        g1 = oracle.bwd(Q[s], K[s], V[s], dO[s], rows[s], cols[s], P, hv, scale)
+        assert np.array_equal(O[s], O1) and np.array_equal(LSE[s], LSE1)
+        for a, b1 in zip((dQ, dK, dV), g1):
+            assert np.array_equal(a[s], b1)
+
+
 # ---------------------------------------------------------------- plan
 
 def rank_formula(keys):

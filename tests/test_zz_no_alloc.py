@@ -4,8 +4,9 @@ Some users of the library run where cudaMalloc is not available to them: the sur
 owns the whole device, or an allocation (which synchronises the device) would break their latency
 budget.  They get one entry point that brings its scratch with it (a fixed array inside the
 library).  This test calls it through the C ABI twice in a row, with different inputs, and checks
-each result against the ordinary mate_attn_bwd: the second call shows that whatever the first call
-left in the shared array does not leak into the next result.
+each result against the CPU oracle's analytic backward and against the ordinary mate_attn_bwd: the
+second call shows that whatever the first call left in the shared array does not leak into the
+next result.  A second case runs the fp32 path with another head size.
 
 Collected last on purpose (file name), so that a run stopping at the first failure has already run
 every other test; it also passes alone in a fresh process.
@@ -14,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from tests import helpers as hp
 from workloads import tables
 
@@ -24,33 +26,52 @@ def _inputs(cfg, rows, cols, seed):
     import paper_2109_04312_b200 as m
     vals = tables.make_values(cfg, rows.shape[1], seed)
     Q, K, V, dO = (hp.to_dev(vals[n], cfg.dtype) for n in ("Q", "K", "V", "dO"))
-    return m, Q, K, V, dO
+    return m, vals, Q, K, V, dO
 
 
-def test_noalloc_backward_matches_the_workspace_backward_twice():
-    cfg = tables.CONFIGS["bert"]
-    rows, cols, info = tables.make_structure(cfg, 4321)
+def _check_twice(cfg, rows, cols, seeds):
     import paper_2109_04312_b200 as m
-    plan = m.mate_plan(torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda(), cfg.P,
-                       tables.head_view(cfg), cfg.n_rows, cfg.n_cols)
+    hv = tables.head_view(cfg)
+    plan = m.mate_plan(torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda(), cfg.P, hv)
     atol, rtol = hp.tol(cfg.dtype)
     valid = rows >= 0
-    for call, seed in enumerate((11, 12)):
-        m, Q, K, V, dO = _inputs(cfg, rows, cols, seed)
+    scale = 1.0 / np.sqrt(cfg.d)
+    for call, seed in enumerate(seeds):
+        m, vals, Q, K, V, dO = _inputs(cfg, rows, cols, seed)
         O, LSE = m.mate_attn_fwd(plan, Q, K, V)
-        ref = m.mate_attn_bwd(plan, Q, K, V, O, LSE, dO)
+        lib = m.mate_attn_bwd(plan, Q, K, V, O, LSE, dO)
+        want = oracle.bwd(vals["Q"], vals["K"], vals["V"], vals["dO"], rows, cols, cfg.P, hv, scale)
         # outputs are the caller's; poison them so that unwritten elements would show
         outs = [torch.full_like(Q, float("nan")) for _ in range(3)]
-        before = torch.cuda.memory_allocated()
+        if call == 0:
+            # the first call on a device looks up the address of the built-in array
+            m.mate_attn_bwd_noalloc(plan, Q, K, V, O, LSE, dO, *outs)
+            torch.cuda.synchronize()
+        # free bytes as the driver counts them: an allocation by the library itself would show here
+        # (torch's own counters only see torch's allocator)
+        free_before = torch.cuda.mem_get_info()[0]
         m.mate_attn_bwd_noalloc(plan, Q, K, V, O, LSE, dO, *outs)
-        assert torch.cuda.memory_allocated() == before
         torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
         plan.status()
-        for name, got, want in zip(("dQ", "dK", "dV"), outs, ref):
-            g, w = hp.to_np(got), hp.to_np(want)
-            hp.assert_close(g, w, atol, rtol, "%s, call %d" % (name, call))
+        for name, got, ref, other in zip(("dQ", "dK", "dV"), outs, want, lib):
+            g = hp.to_np(got)
+            hp.assert_close(g, ref, atol, rtol, "%s vs oracle, call %d" % (name, call))
+            hp.assert_close(g, hp.to_np(other), atol, rtol, "%s vs mate_attn_bwd, call %d" % (name, call))
             assert np.all(g[np.broadcast_to(~valid[:, None, :, None], g.shape)] == 0)
     plan.destroy()
+
+
+def test_noalloc_backward_matches_the_oracle_and_the_workspace_backward_twice():
+    cfg = tables.CONFIGS["bert"]
+    rows, cols, info = tables.make_structure(cfg, 4321)
+    _check_twice(cfg, rows, cols, (11, 12))
+
+
+def test_noalloc_backward_fp32_other_head_size():
+    cfg = tables.CONFIGS["tiny"]                      # fp32, d = 16
+    rows, cols, info = tables.make_structure(cfg, 99)
+    _check_twice(cfg, rows, cols, (5, 6))
 
 
 def test_noalloc_backward_rejects_problems_beyond_its_scratch():
