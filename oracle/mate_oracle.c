@@ -25,8 +25,17 @@
  * statement that a radius covering the longest row / column gives back the exact pattern, and by
  * brute-force attention over the sets.  radius = 0 is the exact pattern.
  *
+ * head_view may also name, per head, the head-independent pattern the paper describes for its
+ * closest comparison system (Section 2: attention restricted to the same row and the same column):
+ * value 2, see oracle_mask_sat.  Pinned by token-by-token sets and by "row pattern OR column
+ * pattern".
+ *
+ * oracle_cell_mean is the mean-pooling of token logits per table cell of Section 4.1,
+ * S(c) = avg over the tokens t of cell c of S(t); pinned by a hand-worked example and per-cell loops.
+ *
  * Layouts: Q, K, V, dO, O, dQ, dK, dV are double [B][H][N][d]; LSE is double [B][H][N];
- * row_ids / col_ids are int32 [B][N]; head_view is uint8 [H] (0 = row head, 1 = column head).
+ * row_ids / col_ids are int32 [B][N]; head_view is uint8 [H] (0 = row head, 1 = column head,
+ * 2 = row-or-column).
  */
 #include <math.h>
 #include <stdint.h>
@@ -69,6 +78,23 @@ void oracle_mask(const int32_t *row_ids, const int32_t *col_ids, int N, int P, i
     }
 }
 
+/* The head-independent pattern the paper describes for its closest comparison system (Section 2,
+ * related work: an attention mask restricting attention to tokens of the same row and of the same
+ * column): a table token attends the query/text prefix and every table token that shares its row
+ * OR its column; prefix tokens attend everything; padding as above.  One pattern for all heads. */
+void oracle_mask_sat(const int32_t *row_ids, const int32_t *col_ids, int N, int P, uint8_t *M) {
+    for (int k = 0; k < N; ++k) {
+        int k_valid = row_ids[k] >= 0 && col_ids[k] >= 0;
+        int k_in_Q = k < P;
+        for (int j = 0; j < N; ++j) {
+            int j_valid = row_ids[j] >= 0 && col_ids[j] >= 0;
+            int j_in_Q = j < P;
+            int in_A = k_in_Q || j_in_Q || row_ids[j] == row_ids[k] || col_ids[j] == col_ids[k];
+            M[(size_t)k * N + j] = (uint8_t)(k_valid && j_valid && in_A);
+        }
+    }
+}
+
 void oracle_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P, int view,
                  int max_id, int32_t *perm, int32_t *inv_perm, int32_t *seg_off);
 
@@ -94,13 +120,23 @@ void oracle_mask_bucketed(const int32_t *row_ids, const int32_t *col_ids, int N,
     free(pos);
 }
 
+/* Mask of one pattern id as used in head_view: 0 = row head, 1 = column head (both Section 3, or
+ * their bucketed form when radius > 0), 2 = the head-independent row-OR-column pattern. */
+static void mask_of_pattern(const int32_t *row_ids, const int32_t *col_ids, int N, int P, int pattern,
+                            int radius, uint8_t *M) {
+    if (pattern == 2)
+        oracle_mask_sat(row_ids, col_ids, N, P, M);
+    else
+        oracle_mask_bucketed(row_ids, col_ids, N, P, pattern, radius, M);
+}
+
 /* Number of unmasked (query, key) pairs per (b, h): popcount of the mask. out: int64 [B][H]. */
 void oracle_useful_pairs(const int32_t *row_ids, const int32_t *col_ids, int B, int H, int N, int P,
                          const uint8_t *head_view, int radius, int64_t *out) {
     uint8_t *M = (uint8_t *)malloc((size_t)N * N);
     for (int b = 0; b < B; ++b)
-        for (int view = 0; view < 2; ++view) {
-            oracle_mask_bucketed(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M);
+        for (int view = 0; view < 3; ++view) {
+            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M);
             int64_t c = 0;
             for (size_t i = 0; i < (size_t)N * N; ++i) c += M[i];
             for (int h = 0; h < H; ++h)
@@ -138,13 +174,12 @@ static double fwd_row(const double *q, const double *K, const double *V, const u
 int oracle_fwd(const double *Q, const double *K, const double *V, const int32_t *row_ids,
                const int32_t *col_ids, int B, int H, int N, int d, int P, const uint8_t *head_view,
                double scale, int radius, double *O, double *LSE) {
-    uint8_t *M[2];
-    M[0] = (uint8_t *)malloc((size_t)N * N);
-    M[1] = (uint8_t *)malloc((size_t)N * N);
-    if (!M[0] || !M[1]) return -1;
+    uint8_t *M[3];
+    for (int v = 0; v < 3; ++v) M[v] = (uint8_t *)malloc((size_t)N * N);
+    if (!M[0] || !M[1] || !M[2]) return -1;
     for (int b = 0; b < B; ++b) {
-        for (int view = 0; view < 2; ++view)
-            oracle_mask_bucketed(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M[view]);
+        for (int view = 0; view < 3; ++view)
+            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M[view]);
 #pragma omp parallel
         {
             double *s = (double *)malloc(sizeof(double) * (size_t)N);
@@ -159,8 +194,7 @@ int oracle_fwd(const double *Q, const double *K, const double *V, const int32_t 
             free(s);
         }
     }
-    free(M[0]);
-    free(M[1]);
+    for (int v = 0; v < 3; ++v) free(M[v]);
     return 0;
 }
 
@@ -175,15 +209,14 @@ int oracle_fwd(const double *Q, const double *K, const double *V, const int32_t 
 int oracle_bwd(const double *Q, const double *K, const double *V, const double *dO,
                const int32_t *row_ids, const int32_t *col_ids, int B, int H, int N, int d, int P,
                const uint8_t *head_view, double scale, int radius, double *dQ, double *dK, double *dV) {
-    uint8_t *M[2];
-    M[0] = (uint8_t *)malloc((size_t)N * N);
-    M[1] = (uint8_t *)malloc((size_t)N * N);
+    uint8_t *M[3];
+    for (int v = 0; v < 3; ++v) M[v] = (uint8_t *)malloc((size_t)N * N);
     double *LSE = (double *)malloc(sizeof(double) * (size_t)H * N);
     double *D = (double *)malloc(sizeof(double) * (size_t)H * N);
-    if (!M[0] || !M[1] || !LSE || !D) return -1;
+    if (!M[0] || !M[1] || !M[2] || !LSE || !D) return -1;
     for (int b = 0; b < B; ++b) {
-        for (int view = 0; view < 2; ++view)
-            oracle_mask_bucketed(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M[view]);
+        for (int view = 0; view < 3; ++view)
+            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M[view]);
         /* pass 1, one query row at a time: LSE_k, D_k, dQ_k */
 #pragma omp parallel
         {
@@ -241,8 +274,7 @@ int oracle_bwd(const double *Q, const double *K, const double *V, const double *
                 }
             }
     }
-    free(M[0]);
-    free(M[1]);
+    for (int v = 0; v < 3; ++v) free(M[v]);
     free(LSE);
     free(D);
     return 0;
@@ -296,4 +328,26 @@ void oracle_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, i
         }
     }
     free(keys);
+}
+
+/* Mean-pooling of per-token logits over the tokens of each table cell (Section 4.1:
+ * S(c) = avg_{t in c} S(t)).  A cell is the set of table tokens (positions >= P with valid ids)
+ * that share a (row id, column id) pair.  mean: double [B][max_row_id+1][max_col_id+1], count:
+ * int32 of the same shape; a pair that no token carries gets count 0 and mean 0. */
+void oracle_cell_mean(const double *logits, const int32_t *row_ids, const int32_t *col_ids, int B, int N,
+                      int P, int max_row_id, int max_col_id, double *mean, int32_t *count) {
+    const int R = max_row_id + 1, Cn = max_col_id + 1;
+    for (int b = 0; b < B; ++b)
+        for (int r = 0; r < R; ++r)
+            for (int c = 0; c < Cn; ++c) {
+                double sum = 0.0;
+                int32_t n = 0;
+                for (int t = P; t < N; ++t)
+                    if (row_ids[(size_t)b * N + t] == r && col_ids[(size_t)b * N + t] == c) {
+                        sum += logits[(size_t)b * N + t];
+                        ++n;
+                    }
+                mean[((size_t)b * R + r) * Cn + c] = n ? sum / n : 0.0;
+                count[((size_t)b * R + r) * Cn + c] = n;
+            }
 }

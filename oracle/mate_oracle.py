@@ -51,6 +51,28 @@ def mask(row_ids, col_ids, P, view, radius=0):
     return M
 
 
+def mask_sat(row_ids, col_ids, P):
+    """Head-independent pattern of Section 2 (same row OR same column, plus the prefix): uint8 [N, N]."""
+    r, c = _i32(row_ids).reshape(-1), _i32(col_ids).reshape(-1)
+    N = r.shape[0]
+    M = np.empty((N, N), dtype=np.uint8)
+    _load().oracle_mask_sat(_p(r), _p(c), C.c_int(N), C.c_int(P), _p(M))
+    return M
+
+
+def cell_mean(logits, row_ids, col_ids, P, max_row_id, max_col_id):
+    """Mean of the token logits per table cell (Section 4.1).  Returns mean f64 and count int32,
+    both [B, max_row_id+1, max_col_id+1]."""
+    x, r, c = _f64(logits), _i32(row_ids), _i32(col_ids)
+    B, N = r.shape
+    assert x.shape == (B, N)
+    mean = np.empty((B, max_row_id + 1, max_col_id + 1), dtype=np.float64)
+    cnt = np.empty((B, max_row_id + 1, max_col_id + 1), dtype=np.int32)
+    _load().oracle_cell_mean(_p(x), _p(r), _p(c), C.c_int(B), C.c_int(N), C.c_int(P), C.c_int(max_row_id),
+                             C.c_int(max_col_id), _p(mean), _p(cnt))
+    return mean, cnt
+
+
 def useful_pairs(row_ids, col_ids, P, head_view, radius=0):
     r, c, hv = _i32(row_ids), _i32(col_ids), _u8(head_view)
     B, N = r.shape
