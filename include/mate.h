@@ -112,6 +112,22 @@ int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int 
                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
                      void *stream, mate_plan_t **out);
 
+/* Plan of the head-independent pattern that the paper describes for its closest comparison system
+ * (Section 2, related work: attention restricted to the tokens of the same row and of the same
+ * column; one pattern for all heads): a table token attends the prefix and every table token that
+ * shares its row id OR its column id; prefix tokens attend every non-padding position; padding as
+ * for mate_plan.  The pattern is evaluated exactly, in three passes of the ordinary kernels over
+ * disjoint key sets -- (prefix and own row), (rest of the own column in front of the own cell),
+ * (rest of the column behind it) -- whose outputs are merged through their logsumexps and whose
+ * gradients are summed; mate_attn_workspace_bytes accounts for the passes' intermediate results.
+ * The returned plan is used with mate_attn_fwd / mate_attn_bwd like any other (all H heads share
+ * the pattern); mate_plan_get returns the row / column orders of mate_plan; mate_plan_useful_pairs
+ * counts the pattern's pairs.  mate_attn_bwd_noalloc does not take such a plan
+ * (MATE_ERR_UNSUPPORTED).  Arguments, ownership and errors as for mate_plan;
+ * (max_row_id + 1) * (max_col_id + 1) must not exceed 2^28. */
+int mate_plan_sat(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len, int H,
+                  int max_row_id, int max_col_id, void *stream, mate_plan_t **out);
+
 /* Copies one view's order to HOST arrays (any pointer may be null to skip it):
  *   perm      int32 [B, N]          perm[b][t] = original position of the t-th token of the view
  *   inv_perm  int32 [B, N]          inverse of perm
@@ -158,6 +174,20 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
                   const void *O, const float *LSE, const void *dO, int d, int dtype, float scale,
                   void *dQ, void *dK, void *dV, void *workspace, size_t workspace_bytes,
                   unsigned flags, void *stream);
+
+/* Per-cell mean of token scores (cell-selection stage, Section 4.1: the score of a cell is the
+ * mean of the scores of its tokens, S(c) = avg_{t in c} S(t)).  A cell is the set of table tokens
+ * (positions behind the prefix, non-negative ids) that share a (row id, column id) pair.
+ *   logits   float32 [B, N], one score per token (prefix and padding positions are ignored)
+ *   col_ids  the int32 [B, N] column ids the plan was made from
+ *   mean     float32 [B, max_row_id + 1, max_col_id + 1], fully overwritten; 0 where no token
+ *            carries the pair
+ *   count    int32, same shape, tokens per cell; may be null
+ * Uses the row view of the plan (a row's tokens are contiguous there).  The sum of a cell runs
+ * over its tokens in original order, so the result is the same on every launch.  Asynchronous on
+ * `stream`; no workspace. */
+int mate_cell_mean(const mate_plan_t *plan, const float *logits, const int32_t *col_ids, float *mean,
+                   int32_t *count, void *stream);
 
 /* Backward for callers that cannot allocate device memory.  (The paper has no counterpart: this
  * entry point exists for the library's users, not for the method.)

@@ -44,6 +44,8 @@ def _load():
     lib.mate_plan_bucketed.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_varlen.restype = i32
     lib.mate_plan_varlen.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
+    lib.mate_plan_sat.restype = i32
+    lib.mate_plan_sat.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_get.restype = i32
     lib.mate_plan_get.argtypes = [vp, i32, vp, vp, vp]
     lib.mate_plan_useful_pairs.restype = i32
@@ -58,6 +60,8 @@ def _load():
     lib.mate_attn_fwd.argtypes = [vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, sz, u32, vp]
     lib.mate_attn_bwd.restype = i32
     lib.mate_attn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, vp, sz, u32, vp]
+    lib.mate_cell_mean.restype = i32
+    lib.mate_cell_mean.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.mate_attn_bwd_noalloc.restype = i32
     lib.mate_attn_bwd_noalloc.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp, vp, vp, vp]
     _lib = lib
@@ -176,6 +180,24 @@ def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_
     return Plan(handle, B, N, prefix_len, int(hv.shape[0]), int(max_row_id), int(max_col_id), row_ids.device)
 
 
+def mate_plan_sat(row_ids, col_ids, prefix_len, n_heads, max_row_id=None, max_col_id=None) -> Plan:
+    """Plan of the head-independent row-or-column pattern (see mate_plan_sat in mate.h)."""
+    if row_ids.dtype != torch.int32 or col_ids.dtype != torch.int32 or row_ids.shape != col_ids.shape \
+            or row_ids.dim() != 2:
+        raise ValueError("row_ids / col_ids must be int32 tensors of the same [B, N] shape")
+    B, N = row_ids.shape
+    if max_row_id is None:
+        max_row_id = max(int(row_ids.max().item()), 0)
+    if max_col_id is None:
+        max_col_id = max(int(col_ids.max().item()), 0)
+    handle = C.c_void_p()
+    with torch.cuda.device(row_ids.device):
+        _check(_load().mate_plan_sat(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N, int(prefix_len),
+                                     int(n_heads), int(max_row_id), int(max_col_id), _stream(), C.byref(handle)),
+               "mate_plan_sat")
+    return Plan(handle, B, N, prefix_len, int(n_heads), int(max_row_id), int(max_col_id), row_ids.device)
+
+
 def mate_attn_workspace_bytes(plan, d, dtype, impl=IMPL_AUTO):
     f, b = C.c_size_t(0), C.c_size_t(0)
     _check(_load().mate_attn_workspace_bytes(plan._h, int(d), dtype, impl, C.byref(f), C.byref(b)),
@@ -236,6 +258,23 @@ def mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale=None, impl=IMPL_AUTO, workspa
                                      ws.numel() if ws is not None else 0, impl, _stream()),
                "mate_attn_bwd")
     return dQ, dK, dV
+
+
+def mate_cell_mean(plan, logits, col_ids, want_count=True):
+    """Mean of the token logits per table cell (see mate_cell_mean in mate.h).  logits: float32 [B, N];
+    col_ids: the int32 [B, N] tensor the plan was made from.  Returns (mean, count) of shape
+    [B, max_row_id + 1, max_col_id + 1] (count is None when not wanted)."""
+    if logits.dtype != torch.float32 or tuple(logits.shape) != (plan.B, plan.N):
+        raise ValueError("logits must be a float32 [B, N] tensor")
+    if col_ids.dtype != torch.int32 or tuple(col_ids.shape) != (plan.B, plan.N):
+        raise ValueError("col_ids must be the int32 [B, N] tensor given to mate_plan")
+    shape = (plan.B, plan.max_id[0] + 1, plan.max_id[1] + 1)
+    mean = torch.empty(shape, dtype=torch.float32, device=logits.device)
+    count = torch.empty(shape, dtype=torch.int32, device=logits.device) if want_count else None
+    with torch.cuda.device(logits.device):
+        _check(_load().mate_cell_mean(plan._h, _dev(logits, "logits"), _dev(col_ids, "col_ids"), _dev(mean, "mean"),
+                                      _dev(count, "count") if want_count else None, _stream()), "mate_cell_mean")
+    return mean, count
 
 
 def mate_attn_bwd_noalloc(plan, Q, K, V, O, LSE, dO, dQ, dK, dV, scale=None):

@@ -70,15 +70,22 @@ struct UnitCost {
 struct RowBounds {
     const int32_t *so;
     int S, P, radius;
+    int mode = mate::kBoundsOwn, group = 1;
     int seg_of(int t) const { return (int)(std::upper_bound(so, so + S, t) - so) - 1; }
     int lo(int t) const {
-        const int l = so[seg_of(t)];
+        const int id = seg_of(t);
+        int l = so[id];
+        if (mode == mate::kBoundsBefore) l = so[id / group * group];
+        if (mode == mate::kBoundsAfter) l = so[id + 1];
         if (radius <= 0) return l;
         const int64_t bk = (t - P) / radius;
         return (int)std::max<int64_t>(l, P + (bk - 1) * radius);
     }
     int hi(int t) const {
-        const int h = so[seg_of(t) + 1];
+        const int id = seg_of(t);
+        int h = so[id + 1];
+        if (mode == mate::kBoundsBefore) h = so[id];
+        if (mode == mate::kBoundsAfter) h = so[std::min((id / group + 1) * group, S - 1)];
         if (radius <= 0) return h;
         const int64_t bk = (t - P) / radius;
         return (int)std::min<int64_t>(h, P + (bk + 2) * radius);
@@ -120,7 +127,7 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
             const int nv = pl->n_valid[b];
             const int P = pl->prefix[b];
-            const RowBounds rb{so, S, P, pl->radius};
+            const RowBounds rb{so, S, P, pl->radius, pl->bounds_mode, pl->group};
             std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
             for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
                 FwdUnit u{};
@@ -204,8 +211,8 @@ int build_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
     pl->bwd_units.clear();
     for (const UnitCost &uc : all) pl->bwd_units.push_back(uc.u);
     pl->n_bwd_units = (int)pl->bwd_units.size();
-    const int64_t share = std::max<int64_t>(total_cost / n_ctas, 1);
-    // forward: long prefix units split
+    // forward: long prefix units split; the forward kernel runs several CTAs per SM
+    const int64_t share = std::max<int64_t>(total_cost / ((int64_t)n_ctas * mate::tc_fwd_ctas_per_sm()), 1);
     make_units(pl, seg_off_host, share, all, &n_slots, &ws_bytes, &total_cost);
     pl->fwd_units.clear();
     for (const UnitCost &uc : all) pl->fwd_units.push_back(uc.u);
@@ -256,6 +263,8 @@ const char *mate_status_string(int status) {
 
 int mate_plan_destroy(mate_plan_t *plan) {
     if (!plan) return MATE_OK;
+    for (int s = 0; s < 2; ++s) mate_plan_destroy(plan->sub[s]);
+    if (plan->pair_ids_dev) cudaFree(plan->pair_ids_dev);
     if (plan->dev_block) cudaFree(plan->dev_block);
     if (plan->work_block) cudaFree(plan->work_block);
     delete plan;
@@ -279,9 +288,58 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
                             stream, out);
 }
 
+static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
+                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius, int bounds_mode,
+                      int group, void *stream, mate_plan_t **out);
+
 int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
                      void *stream, mate_plan_t **out) {
+    return build_plan(row_ids, col_ids, B, N, prefix_len, head_view, H, max_row_id, max_col_id, radius,
+                      mate::kBoundsOwn, 1, stream, out);
+}
+
+/* The head-independent pattern: three passes over plans the ordinary kernels can run (see mate.h).
+ *   main plan  every head a row head: prefix rows against everything, table rows against the prefix
+ *              and their own row (which holds their own cell)
+ *   sub[0]     ids = (column, row) pairs, column-major, prefix treated as padding: table rows against
+ *              the cells of their column in front of their own cell
+ *   sub[1]     the same behind their own cell
+ * The three key sets of a row are disjoint and their union is the pattern. */
+int mate_plan_sat(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len, int H,
+                  int max_row_id, int max_col_id, void *stream, mate_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!out || B <= 0 || H <= 0 || max_row_id < 0 || max_col_id < 0) return MATE_ERR_INVALID_ARG;
+    if ((long long)(max_row_id + 1) * (max_col_id + 1) > (1ll << 28)) return MATE_ERR_UNSUPPORTED;
+    const std::vector<int32_t> prefix((size_t)B, prefix_len), zero((size_t)B, 0);
+    const std::vector<uint8_t> rows_only((size_t)H, 0), cols_only((size_t)H, 1);
+    mate_plan_t *pl = nullptr;
+    int rc = build_plan(row_ids, col_ids, B, N, prefix.data(), rows_only.data(), H, max_row_id, max_col_id, 0,
+                        mate::kBoundsOwn, 1, stream, &pl);
+    if (rc != MATE_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int n_row_ids = max_row_id + 1, max_pair = n_row_ids * (max_col_id + 1) - 1;
+    bool ok = cudaMalloc(&pl->pair_ids_dev, sizeof(int32_t) * (size_t)B * N) == cudaSuccess;
+    ok = ok && mate::launch_pair_ids(row_ids, col_ids, B, N, pl->prefix_dev, n_row_ids, pl->pair_ids_dev, st) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        mate_plan_destroy(pl);
+        return MATE_ERR_NOMEM;
+    }
+    for (int s = 0; s < 2 && rc == MATE_OK; ++s)
+        rc = build_plan(pl->pair_ids_dev, pl->pair_ids_dev, B, N, zero.data(), cols_only.data(), H, max_pair, max_pair, 0,
+                        s == 0 ? mate::kBoundsBefore : mate::kBoundsAfter, n_row_ids, stream, &pl->sub[s]);
+    if (rc != MATE_OK) {
+        mate_plan_destroy(pl);
+        return rc;
+    }
+    *out = pl;
+    return MATE_OK;
+}
+
+static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
+                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius, int bounds_mode,
+                      int group, void *stream, mate_plan_t **out) {
     if (out) *out = nullptr;
     if (radius < 0) return MATE_ERR_INVALID_ARG;
     if (!row_ids || !col_ids || !head_view || !out || !prefix_len) return MATE_ERR_INVALID_ARG;
@@ -302,6 +360,8 @@ int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int 
     pl->prefix.assign(prefix_len, prefix_len + B);
     pl->H = H;
     pl->radius = radius;
+    pl->bounds_mode = bounds_mode;
+    pl->group = std::max(group, 1);
     pl->head_view.assign(head_view, head_view + H);
     pl->view[0].max_id = max_row_id;
     pl->view[1].max_id = max_col_id;
@@ -334,7 +394,7 @@ int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int 
                                st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(pl->prefix_dev, pl->prefix.data(), B * sizeof(int32_t), cudaMemcpyHostToDevice,
                                st) == cudaSuccess;
-    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, pl->prefix_dev, radius, pl->view[0], pl->view[1],
+    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, pl->prefix_dev, radius, bounds_mode, pl->group, pl->view[0], pl->view[1],
                                          pl->n_valid_dev, pl->status_dev, st) == cudaSuccess;
     for (int v = 0; v < 2 && ok; ++v) {
         seg_off_host[v].resize((size_t)B * (pl->view[v].max_id + 2));
@@ -363,8 +423,8 @@ int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int 
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
             const int P = pl->prefix[b];
             int64_t c = (int64_t)P * pl->n_valid[b];
-            if (radius > 0) {
-                const RowBounds rb{so, S, P, radius};
+            if (radius > 0 || pl->bounds_mode != mate::kBoundsOwn) {
+                const RowBounds rb{so, S, P, radius, pl->bounds_mode, pl->group};
                 for (int t = P; t < pl->n_valid[b]; ++t) c += P + rb.hi(t) - rb.lo(t);
             } else {
                 for (int s = 0; s + 1 < S; ++s) {
@@ -415,20 +475,32 @@ int mate_plan_get(const mate_plan_t *plan, int view, int32_t *perm, int32_t *inv
 int mate_plan_useful_pairs(const mate_plan_t *plan, int64_t *pairs) {
     if (!plan || !pairs) return MATE_ERR_INVALID_ARG;
     for (int b = 0; b < plan->B; ++b)
-        for (int h = 0; h < plan->H; ++h)
-            pairs[(size_t)b * plan->H + h] = plan->pairs[(size_t)b * 2 + plan->head_view[h]];
+        for (int h = 0; h < plan->H; ++h) {
+            int64_t c = plan->pairs[(size_t)b * 2 + plan->head_view[h]];
+            for (int s = 0; s < 2; ++s)
+                if (plan->sub[s]) c += plan->sub[s]->pairs[(size_t)b * 2 + 1];
+            pairs[(size_t)b * plan->H + h] = c;
+        }
     return MATE_OK;
 }
 
 int mate_plan_status(const mate_plan_t *plan, void *stream) {
     if (!plan) return MATE_ERR_INVALID_ARG;
+    for (int s = 0; s < 2; ++s)
+        if (plan->sub[s]) {
+            const int rc = mate_plan_status(plan->sub[s], stream);
+            if (rc != MATE_OK) return rc;
+        }
     cudaStream_t st = (cudaStream_t)stream;
     int32_t s[4] = {0, 0, 0, 0};
     if (cudaMemcpyAsync(s, plan->status_dev, sizeof(s), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaMemsetAsync(plan->status_dev + 1, 0, sizeof(int32_t), st) != cudaSuccess ||
+        cudaMemsetAsync(plan->status_dev + 1, 0, 2 * sizeof(int32_t), st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess)
         return MATE_ERR_CUDA;
     if (s[1] != 0) {
+        if (getenv("MATE_LOG"))
+            fprintf(stderr, "[mate] a bounded wait expired: barrier slot %d, parity %d, warp %d\n", (s[2] >> 8) & 0xff,
+                    (s[2] >> 7) & 1, s[2] & 0x7f);
         // a kernel that gave up may have left the scheduling and arrival counters half way
         if (cudaMemsetAsync(plan->fwd_counters_dev, 0,
                             sizeof(int32_t) * (mate::kSchedWords + 8 * (size_t)plan->n_fwd_slots), st) != cudaSuccess ||
@@ -459,14 +531,40 @@ static int check_common(const mate_plan_t *plan, int d, int dtype, unsigned flag
     return MATE_OK;
 }
 
+// Scratch of one pass (the ordinary kernels) and of a whole call.  For a row-or-column plan the call
+// holds, behind the passes' own scratch (the passes run one after the other and share it), the
+// outputs of the two extra passes: forward 2 x (O + LSE), backward 2 x (dQ, dK, dV).
+static size_t pass_fwd_bytes(const mate_plan_t *plan, int d, bool use_tc) {
+    size_t n = use_tc ? mate::tc_fwd_workspace(plan, d) : 0;
+    for (int s = 0; s < 2; ++s)
+        if (plan->sub[s]) n = std::max(n, use_tc ? mate::tc_fwd_workspace(plan->sub[s], d) : (size_t)0);
+    return align_up(n, 256);
+}
+static size_t pass_bwd_bytes(const mate_plan_t *plan, bool use_tc) {
+    return align_up(use_tc ? mate::tc_bwd_workspace(plan) : mate::simt_bwd_workspace(plan), 256);
+}
+static size_t elem_bytes(int dtype) { return dtype == MATE_F32 ? 4 : 2; }
+
 int mate_attn_workspace_bytes(const mate_plan_t *plan, int d, int dtype, unsigned flags,
                               size_t *fwd_bytes, size_t *bwd_bytes) {
     bool use_tc = false;
     int rc = check_common(plan, d, dtype, flags, &use_tc);
     if (rc != MATE_OK) return rc;
-    if (fwd_bytes) *fwd_bytes = use_tc ? mate::tc_fwd_workspace(plan, d) : 0;
-    if (bwd_bytes) *bwd_bytes = use_tc ? mate::tc_bwd_workspace(plan) : mate::simt_bwd_workspace(plan);
+    const size_t rows = (size_t)plan->B * plan->H * plan->N;
+    size_t f = pass_fwd_bytes(plan, d, use_tc), b = pass_bwd_bytes(plan, use_tc);
+    if (plan->sub[0]) {
+        f += 2 * (align_up(rows * d * elem_bytes(dtype), 256) + align_up(rows * sizeof(float), 256));
+        b += 6 * align_up(rows * d * elem_bytes(dtype), 256);
+    }
+    if (fwd_bytes) *fwd_bytes = f;
+    if (bwd_bytes) *bwd_bytes = b;
     return MATE_OK;
+}
+
+static int fwd_pass(const mate_plan_t *plan, bool use_tc, const void *Q, const void *K, const void *V, int d, int dtype,
+                    float scale, void *O, float *LSE, void *ws, cudaStream_t st) {
+    if (use_tc) return mate::tc_fwd(plan, Q, K, V, scale, O, LSE, ws, st);
+    return mate::simt_fwd(plan, Q, K, V, d, dtype, scale, O, LSE, st);
 }
 
 int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d,
@@ -485,13 +583,34 @@ int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const v
         if ((flags & 3u) == MATE_IMPL_TCGEN05) return MATE_ERR_UNSUPPORTED;
         use_tc = false;
     }
-    if (use_tc) {
-        const size_t need = mate::tc_fwd_workspace(plan, d);
-        if (need > 0 && (!workspace || workspace_bytes < need)) return MATE_ERR_WORKSPACE;
-        if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MATE_ERR_ALIGNMENT;
-        return mate::tc_fwd(plan, Q, K, V, scale, O, LSE, workspace, st);
+    size_t need = 0;
+    mate_attn_workspace_bytes(plan, d, dtype, use_tc ? MATE_IMPL_TCGEN05 : MATE_IMPL_SIMT, &need, nullptr);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return MATE_ERR_WORKSPACE;
+    if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MATE_ERR_ALIGNMENT;
+    rc = fwd_pass(plan, use_tc, Q, K, V, d, dtype, scale, O, LSE, workspace, st);
+    if (rc != MATE_OK || !plan->sub[0]) return rc;
+    // row-or-column pattern: the two passes over the rest of the column, then the merge
+    const size_t rows = (size_t)plan->B * plan->H * plan->N;
+    const size_t o_bytes = align_up(rows * d * elem_bytes(dtype), 256), l_bytes = align_up(rows * sizeof(float), 256);
+    char *w = (char *)workspace + pass_fwd_bytes(plan, d, use_tc);
+    void *Os[2];
+    float *Ls[2];
+    for (int s = 0; s < 2; ++s) {
+        Os[s] = w;
+        Ls[s] = (float *)(w + o_bytes);
+        w += o_bytes + l_bytes;
+        rc = fwd_pass(plan->sub[s], use_tc, Q, K, V, d, dtype, scale, Os[s], Ls[s], workspace, st);
+        if (rc != MATE_OK) return rc;
     }
-    return mate::simt_fwd(plan, Q, K, V, d, dtype, scale, O, LSE, st);
+    return mate::launch_merge_passes(O, LSE, Os[0], Ls[0], Os[1], Ls[1], rows, d, dtype, st) == cudaSuccess ? MATE_OK
+                                                                                                           : MATE_ERR_CUDA;
+}
+
+static int bwd_pass(const mate_plan_t *plan, bool use_tc, const void *Q, const void *K, const void *V, const void *O,
+                    const float *LSE, const void *dO, int d, int dtype, float scale, void *dQ, void *dK, void *dV, void *ws,
+                    cudaStream_t st) {
+    if (use_tc) return mate::tc_bwd(plan, Q, K, V, O, LSE, dO, scale, dQ, dK, dV, ws, st);
+    return mate::simt_bwd(plan, Q, K, V, O, LSE, dO, d, dtype, scale, dQ, dK, dV, ws, st);
 }
 
 int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
@@ -506,13 +625,30 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     const void *ptrs[] = {Q, K, V, O, LSE, dO, dQ, dK, dV};
     for (const void *p : ptrs)
         if (!aligned16(p)) return MATE_ERR_ALIGNMENT;
-    const size_t need = use_tc ? mate::tc_bwd_workspace(plan) : mate::simt_bwd_workspace(plan);
+    size_t need = 0;
+    mate_attn_workspace_bytes(plan, d, dtype, use_tc ? MATE_IMPL_TCGEN05 : MATE_IMPL_SIMT, nullptr, &need);
     if (!workspace || workspace_bytes < need) return MATE_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) return MATE_ERR_ALIGNMENT;
-    if (use_tc)
-        return mate::tc_bwd(plan, Q, K, V, O, LSE, dO, scale, dQ, dK, dV, workspace, (cudaStream_t)stream);
-    return mate::simt_bwd(plan, Q, K, V, O, LSE, dO, d, dtype, scale, dQ, dK, dV, workspace,
-                          (cudaStream_t)stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    rc = bwd_pass(plan, use_tc, Q, K, V, O, LSE, dO, d, dtype, scale, dQ, dK, dV, workspace, st);
+    if (rc != MATE_OK || !plan->sub[0]) return rc;
+    // Row-or-column pattern.  With the final O and LSE every pass computes the gradient of its own
+    // pairs.  The two column passes are each other's transpose (keys in front of / behind the own
+    // cell), and the kernels take a plan's key ranges for the query side and for the key side alike;
+    // run on both plans and summed, every pair is still counted once on each side.
+    const size_t n = (size_t)plan->B * plan->H * plan->N * d;
+    const size_t g_bytes = align_up(n * elem_bytes(dtype), 256);
+    char *w = (char *)workspace + pass_bwd_bytes(plan, use_tc);
+    void *g[2][3];
+    for (int s = 0; s < 2; ++s) {
+        for (int i = 0; i < 3; ++i, w += g_bytes) g[s][i] = w;
+        rc = bwd_pass(plan->sub[s], use_tc, Q, K, V, O, LSE, dO, d, dtype, scale, g[s][0], g[s][1], g[s][2], workspace, st);
+        if (rc != MATE_OK) return rc;
+    }
+    void *outs[3] = {dQ, dK, dV};
+    for (int i = 0; i < 3; ++i)
+        if (mate::launch_add3(outs[i], g[0][i], g[1][i], n, dtype, st) != cudaSuccess) return MATE_ERR_CUDA;
+    return MATE_OK;
 }
 
 }  // extern "C"

@@ -34,7 +34,7 @@
 namespace mate {
 
 #ifdef MATE_TRACE
-__device__ long long g_trace_bwd[148 * 32];
+__device__ long long g_trace_bwd[kTraceCtas * 32];
 #endif
 
 namespace {
@@ -800,7 +800,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
     }
 
 #ifdef MATE_TRACE
-    if (lane == 0 && (warp == 0 || warp == 4 || warp == kMmaWarp || warp == kLoadWarp0)) {
+    if (lane == 0 && (warp == 0 || warp == 4 || warp == kMmaWarp || warp == kLoadWarp0) && blockIdx.x < kTraceCtas) {
         const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == kMmaWarp ? 2 : 3;
         long long *o = g_trace_bwd + blockIdx.x * 32 + role * 8;
         for (int i = 0; i < 8; ++i) o[i] = tr[i];
@@ -862,8 +862,8 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 }  // namespace mate
 
 #ifdef MATE_TRACE
-// copies the cycle counters of the last backward launch to the host: [148 CTAs][4 roles][8]
+// copies the cycle counters of the last backward launch to the host: [kTraceCtas CTAs][4 roles][8]
 extern "C" int mate_debug_trace_bwd(long long *host_out) {
-    return cudaMemcpyFromSymbol(host_out, mate::g_trace_bwd, sizeof(long long) * 148 * 32) == cudaSuccess ? 0 : -4;
+    return cudaMemcpyFromSymbol(host_out, mate::g_trace_bwd, sizeof(long long) * mate::kTraceCtas * 32) == cudaSuccess ? 0 : -4;
 }
 #endif

@@ -30,7 +30,7 @@
 namespace mate {
 
 #ifdef MATE_TRACE
-__device__ long long g_trace[148 * 32];
+__device__ long long g_trace[kTraceCtas * 32];
 #endif
 
 namespace {
@@ -517,7 +517,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             tc_wait_ld();
 
             if (un.n_parts == 1) {
-                const float inv_l = 1.f / l;
+                const float inv_l = l > 0.f ? 1.f / l : 0.f;  // a row without any key (possible in the passes of the
+                                                               // row-or-column pattern) gives O = 0, LSE = -inf
                 if (row_valid) {
                     uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
 #pragma unroll
@@ -874,7 +875,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
     }
 
 #ifdef MATE_TRACE
-    if (lane == 0 && (warp == 0 || warp == 4 || warp == kMmaWarp || warp == kLoadWarp0)) {  // MMA: half 0's thread
+    if (lane == 0 && (warp == 0 || warp == 4 || warp == kMmaWarp || warp == kLoadWarp0) &&
+        blockIdx.x < kTraceCtas) {  // MMA: half 0's thread
         const int role = warp == 0 ? 0 : warp == 4 ? 1 : warp == kMmaWarp ? 2 : 3;
         long long *o = g_trace + blockIdx.x * 32 + role * 8;
         for (int i = 0; i < 7; ++i) o[i] = tr[i];
@@ -901,11 +903,13 @@ SmemAttrOnce g_smem_attr;
 
 bool tc_supported(int d, int dtype) { return d == 64 && dtype == MATE_BF16; }
 
+int tc_fwd_ctas_per_sm() { return 1; }
+
 size_t tc_fwd_workspace(const mate_plan_t *plan, int) { return plan->fwd_ws_bytes; }
 
 int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, float scale, void *O,
            float *LSE, void *workspace, cudaStream_t stream) {
-    if (!(scale > 0.f)) return MATE_ERR_UNSUPPORTED;  // the row max is taken before scaling
+    if (!(scale > 0.f)) return MATE_ERR_UNSUPPORTED;  // the row max is taken before scaling (the caller falls back)
     if (plan->n_fwd_units == 0) return MATE_OK;
     if (g_smem_attr.ensure((const void *)tc_fwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
     Params p;
@@ -932,8 +936,8 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 }  // namespace mate
 
 #ifdef MATE_TRACE
-// copies the cycle counters of the last forward launch to the host: [148 CTAs][4 roles][8]
+// copies the cycle counters of the last forward launch to the host: [kTraceCtas CTAs][4 roles][8]
 extern "C" int mate_debug_trace(long long *host_out) {
-    return cudaMemcpyFromSymbol(host_out, mate::g_trace, sizeof(long long) * 148 * 32) == cudaSuccess ? 0 : -4;
+    return cudaMemcpyFromSymbol(host_out, mate::g_trace, sizeof(long long) * mate::kTraceCtas * 32) == cudaSuccess ? 0 : -4;
 }
 #endif

@@ -13,6 +13,10 @@ namespace mate {
 constexpr int kTile = 128;       // key columns per tile and query rows per half of a unit
 constexpr int kSchedWords = 8;   // scheduling counters in front of the split-unit counters
 constexpr int kUnitRows = 256;   // query rows per unit of the tensor-core kernels (two halves)
+// what the key range of a table row is made of (plan kernel step 4 and its host twin)
+enum { kBoundsOwn = 0, kBoundsBefore = 1, kBoundsAfter = 2 };
+constexpr int kTraceCtas = 256;  // CTAs whose cycle counters a -DMATE_TRACE build keeps
+constexpr int kTraceEvents = 2048;  // time-stamped events per role of CTA 0 in such a build
 
 // One unit of work of the tensor-core forward: up to 256 consecutive query rows (view order) of one
 // (example, head) -- half 0 = the first 128 rows, half 1 = the rest -- and the key tiles (128 wide)
@@ -58,6 +62,11 @@ struct mate_plan_s {
     std::vector<int32_t> prefix;         // |Q| per example (host copy)
     int32_t *prefix_dev = nullptr;       // [B]
     int radius = 0;                      // > 0: bucketed pattern (Section 3.1), buckets of this many positions
+    int bounds_mode = 0, group = 1;      // key range of a table row (kBounds*), ids per group
+    // row-or-column pattern (mate_plan_sat): this plan is the row pass; sub[0] / sub[1] are the passes
+    // over the rest of the token's column in front of / behind its own cell
+    mate_plan_s *sub[2] = {nullptr, nullptr};
+    int32_t *pair_ids_dev = nullptr;     // ids of the sub-plans (owned by the main plan)
     std::vector<uint8_t> head_view;      // host copy
     uint8_t *head_view_dev = nullptr;    // [H]
     mate::ViewPlan view[2];
@@ -107,8 +116,16 @@ struct SmemAttrOnce {
 
 // plan kernels (mate_plan_kernels.cu)
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,
-                                const int32_t *prefix /* device [B] */, int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
-                                int32_t *status, cudaStream_t stream);
+                                const int32_t *prefix /* device [B] */, int radius, int bounds_mode, int group,
+                                const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid, int32_t *status,
+                                cudaStream_t stream);
+cudaError_t launch_pair_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix,
+                            int n_row_ids, int32_t *out, cudaStream_t stream);
+
+// row-or-column pattern (mate_sat.cu): merge of the passes' outputs, sum of their gradients
+cudaError_t launch_merge_passes(void *O, float *LSE, const void *O1, const float *LSE1, const void *O2, const float *LSE2,
+                                size_t rows, int d, int dtype, cudaStream_t stream);
+cudaError_t launch_add3(void *a, const void *b, const void *c, size_t n, int dtype, cudaStream_t stream);
 
 // SIMT kernels (mate_simt.cu)
 int simt_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d, int dtype,
@@ -120,6 +137,7 @@ int simt_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *
 
 // tensor-core kernels (mate_fwd_tc.cu / mate_bwd_tc.cu)
 bool tc_supported(int d, int dtype);
+int tc_fwd_ctas_per_sm();  // CTAs of the forward kernel per SM (the grid is this times the plan's SM count)
 size_t tc_fwd_workspace(const mate_plan_t *plan, int d);
 size_t tc_bwd_workspace(const mate_plan_t *plan);
 int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, const void *O,
@@ -134,10 +152,20 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 // the tensor-core kernels, per CTA and role, in a local array `tr`.  Profiling aid only; compiled
 // out of the library.
 #ifdef MATE_TRACE
+// event log of CTA 0 (two roles, time-stamped): TR_EV(role, id) in one lane of a warp
+#define TR_EV(role, id)                                                              \
+    do {                                                                             \
+        if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && ev_n < mate::kTraceEvents) { \
+            mate::g_evlog[((role) * mate::kTraceEvents + ev_n) * 2] = (id);            \
+            mate::g_evlog[((role) * mate::kTraceEvents + ev_n) * 2 + 1] = clock64();   \
+            ++ev_n;                                                                  \
+        }                                                                            \
+    } while (0)
 #define TR_T0(var) const long long var = clock64()
 #define TR_ADD(cat, var) tr[cat] += clock64() - (var)
 #define TR_INC(cat) tr[cat] += 1
 #else
+#define TR_EV(role, id)
 #define TR_T0(var)
 #define TR_ADD(cat, var)
 #define TR_INC(cat)

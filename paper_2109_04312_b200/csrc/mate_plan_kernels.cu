@@ -21,7 +21,7 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane) {
 
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N,
-            const int32_t *__restrict__ prefix, int radius,
+            const int32_t *__restrict__ prefix, int radius, int bounds_mode, int group,
             ViewPlan rowv, ViewPlan colv, int32_t *__restrict__ n_valid_out,
             int32_t *__restrict__ status) {
     __shared__ int32_t s_cursor[kSmemIds];
@@ -121,7 +121,9 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
     }
     __syncthreads();
 
-    // 4. per view position: the key range of its own segment.  With a radius (the bucketed form of
+    // 4. per view position: its key range.  Normally its own segment; for the passes of the
+    //    row-or-column pattern, whose ids are (column, row) pairs in groups of `group` ids per
+    //    column, the segments of its group in front of / behind its own.  With a radius (the bucketed form of
     //    Section 3.1: the order behind the prefix is cut into buckets of `radius` positions and a
     //    token sees its own bucket and the two next to it) the range is clipped to those buckets.
     int32_t *seg_lo = vp.seg_lo + (size_t)b * N, *seg_hi = vp.seg_hi + (size_t)b * N;
@@ -133,6 +135,13 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
             int id = ids[perm[t]];
             lo = seg_off[id];
             hi = seg_off[id + 1];
+            if (bounds_mode == kBoundsBefore) {  // the segments of the same group in front of the own one
+                hi = lo;
+                lo = seg_off[id / group * group];
+            } else if (bounds_mode == kBoundsAfter) {  // ... behind the own one
+                lo = hi;
+                hi = seg_off[min((id / group + 1) * group, vp.max_id + 1)];
+            }
             if (radius > 0) {
                 const long long bk = (t - P) / radius;
                 const long long w0 = P + (bk - 1) * radius, w1 = P + (bk + 2) * radius;
@@ -148,11 +157,31 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
 }  // namespace
 
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,
-                                const int32_t *prefix, int radius, const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid,
-                                int32_t *status, cudaStream_t stream) {
+                                const int32_t *prefix, int radius, int bounds_mode, int group, const ViewPlan &rowv,
+                                const ViewPlan &colv, int32_t *n_valid, int32_t *status, cudaStream_t stream) {
     dim3 grid(B, 2);
-    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, prefix, radius, rowv, colv, n_valid,
-                                                   status);
+    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, prefix, radius, bounds_mode, max(group, 1), rowv,
+                                                   colv, n_valid, status);
+    return cudaGetLastError();
+}
+
+namespace {
+// ids of the two extra passes of the row-or-column pattern: (column, row) pairs as one id,
+// column-major, for table tokens; -1 (treated as padding by those passes) for everything else
+__global__ void pair_ids_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, size_t n,
+                                int N, const int32_t *__restrict__ prefix, int n_row_ids, int32_t *__restrict__ out) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int b = (int)(i / N), k = (int)(i % N);
+    const int r = row_ids[i], c = col_ids[i];
+    out[i] = (k >= prefix[b] && r >= 0 && c >= 0) ? c * n_row_ids + r : -1;
+}
+}  // namespace
+
+cudaError_t launch_pair_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix,
+                            int n_row_ids, int32_t *out, cudaStream_t stream) {
+    const size_t n = (size_t)B * N;
+    pair_ids_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(row_ids, col_ids, n, N, prefix, n_row_ids, out);
     return cudaGetLastError();
 }
 

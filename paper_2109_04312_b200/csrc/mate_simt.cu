@@ -126,7 +126,9 @@ simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
             }
         }
     }
-    const float inv_l = 1.f / l;  // every valid row attends at least to itself, so l > 0
+    // a valid row attends at least to itself, except in the passes of the row-or-column pattern,
+    // where a row may have no key at all: O = 0, LSE = -inf
+    const float inv_l = l > 0.f ? 1.f / l : 0.f;
 #pragma unroll
     for (int i = 0; i < kAccPerLane; ++i) {
         const int e = lane + 32 * i;
@@ -314,6 +316,7 @@ extern "C" int mate_attn_bwd_noalloc(const mate_plan_t *plan, const void *Q, con
     const void *ptrs[] = {Q, K, V, O, LSE, dO, dQ, dK, dV};
     for (const void *p : ptrs)
         if (reinterpret_cast<uintptr_t>(p) & 15u) return MATE_ERR_ALIGNMENT;
+    if (plan->sub[0]) return MATE_ERR_UNSUPPORTED;  // row-or-column plans need the three-pass path
     const size_t rows = (size_t)plan->B * plan->H * plan->N;
     if (rows > mate::kNoAllocMaxRows) return MATE_ERR_TOO_LARGE;
 
