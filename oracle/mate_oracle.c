@@ -18,10 +18,10 @@
  * Parity of these conventions is unpinned by the paper; every arithmetic function below is pinned
  * by closed forms, brute force and finite differences in the CPU test-suite.
  *
- * A radius argument > 0 selects the bucketed approximation of Section 3.1 / Appendix D with the
- * global part G = the prefix: in a head's own order the positions after the prefix are cut into
- * buckets of `radius`, and a table token keeps, of A^i_k, the prefix and the keys whose bucket is
- * its own or adjacent.  Pinned by a token-by-token construction of those sets, by the paper's
+ * A radius argument > 0 selects the bucketed approximation of Section 3.1 / Appendix D: in a
+ * head's own order the first G positions (G >= P, the global section) attend and are attended by
+ * everything, the positions behind them are cut into buckets of `radius`, and such a token keeps,
+ * of A^i_k, the global section and the keys whose bucket is its own or adjacent.  Pinned by a token-by-token construction of those sets, by the paper's
  * statement that a radius covering the longest row / column gives back the exact pattern, and by
  * brute-force attention over the sets.  radius = 0 is the exact pattern.
  *
@@ -98,23 +98,32 @@ void oracle_mask_sat(const int32_t *row_ids, const int32_t *col_ids, int N, int 
 void oracle_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int P, int view,
                  int max_id, int32_t *perm, int32_t *inv_perm, int32_t *seg_off);
 
-/* Bucketed pattern (Section 3.1, Appendix D; G = the prefix, bucket length = radius).  Every head
- * orders the tokens its own way (oracle_plan); the positions of that order behind the prefix are
- * cut into buckets of `radius`; a table token attends the global part and, within A_k, the tokens
- * of its own bucket and of the two adjacent buckets.  Global (prefix) tokens keep their full sets.
- * radius <= 0: the exact pattern. */
+/* Bucketed pattern (Section 3.1, Appendix D).  Every head orders the tokens its own way
+ * (oracle_plan).  The first G positions of that order are the global section: they attend every
+ * position and every position attends them (G >= P: the prefix, and, when G is larger, the table
+ * tokens that come first in the head's order; Appendix A.2 uses G = 116).  The positions behind it
+ * are cut into buckets of `radius`; such a token attends the global section and, within A_k, the
+ * tokens of its own bucket and of the two adjacent buckets.  radius <= 0: the exact pattern (G is
+ * then without effect); G < P is read as G = P. */
 void oracle_mask_bucketed(const int32_t *row_ids, const int32_t *col_ids, int N, int P, int view,
-                          int radius, uint8_t *M) {
+                          int radius, int G, uint8_t *M) {
     oracle_mask(row_ids, col_ids, N, P, view, M);
     if (radius <= 0) return;
+    if (G < P) G = P;
+    const int32_t *id = view == 0 ? row_ids : col_ids;
     int32_t *perm = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
     int32_t *pos = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
     int32_t seg[2];
     oracle_plan(row_ids, col_ids, 1, N, P, view, 0, perm, pos, seg);
-    for (int k = P; k < N; ++k)
-        for (int j = P; j < N; ++j) {
-            int bucket_k = (pos[k] - P) / radius, bucket_j = (pos[j] - P) / radius;
-            if (abs(bucket_k - bucket_j) > 1) M[(size_t)k * N + j] = 0;
+    for (int k = 0; k < N; ++k)
+        for (int j = 0; j < N; ++j) {
+            if (id[k] < 0 || id[j] < 0) continue; /* padding stays excluded */
+            if (pos[k] < G || pos[j] < G) {
+                M[(size_t)k * N + j] = 1; /* to and from the global section */
+            } else {
+                int bucket_k = (pos[k] - G) / radius, bucket_j = (pos[j] - G) / radius;
+                if (abs(bucket_k - bucket_j) > 1) M[(size_t)k * N + j] = 0;
+            }
         }
     free(perm);
     free(pos);
@@ -123,20 +132,20 @@ void oracle_mask_bucketed(const int32_t *row_ids, const int32_t *col_ids, int N,
 /* Mask of one pattern id as used in head_view: 0 = row head, 1 = column head (both Section 3, or
  * their bucketed form when radius > 0), 2 = the head-independent row-OR-column pattern. */
 static void mask_of_pattern(const int32_t *row_ids, const int32_t *col_ids, int N, int P, int pattern,
-                            int radius, uint8_t *M) {
+                            int radius, int G, uint8_t *M) {
     if (pattern == 2)
         oracle_mask_sat(row_ids, col_ids, N, P, M);
     else
-        oracle_mask_bucketed(row_ids, col_ids, N, P, pattern, radius, M);
+        oracle_mask_bucketed(row_ids, col_ids, N, P, pattern, radius, G, M);
 }
 
 /* Number of unmasked (query, key) pairs per (b, h): popcount of the mask. out: int64 [B][H]. */
 void oracle_useful_pairs(const int32_t *row_ids, const int32_t *col_ids, int B, int H, int N, int P,
-                         const uint8_t *head_view, int radius, int64_t *out) {
+                         const uint8_t *head_view, int radius, int G, int64_t *out) {
     uint8_t *M = (uint8_t *)malloc((size_t)N * N);
     for (int b = 0; b < B; ++b)
         for (int view = 0; view < 3; ++view) {
-            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M);
+            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, G, M);
             int64_t c = 0;
             for (size_t i = 0; i < (size_t)N * N; ++i) c += M[i];
             for (int h = 0; h < H; ++h)
@@ -173,13 +182,13 @@ static double fwd_row(const double *q, const double *K, const double *V, const u
 
 int oracle_fwd(const double *Q, const double *K, const double *V, const int32_t *row_ids,
                const int32_t *col_ids, int B, int H, int N, int d, int P, const uint8_t *head_view,
-               double scale, int radius, double *O, double *LSE) {
+               double scale, int radius, int G, double *O, double *LSE) {
     uint8_t *M[3];
     for (int v = 0; v < 3; ++v) M[v] = (uint8_t *)malloc((size_t)N * N);
     if (!M[0] || !M[1] || !M[2]) return -1;
     for (int b = 0; b < B; ++b) {
         for (int view = 0; view < 3; ++view)
-            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M[view]);
+            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, G, M[view]);
 #pragma omp parallel
         {
             double *s = (double *)malloc(sizeof(double) * (size_t)N);
@@ -208,7 +217,7 @@ int oracle_fwd(const double *Q, const double *K, const double *V, const int32_t 
  * O and LSE are recomputed here from Q, K, V, so the result depends on no forward output. */
 int oracle_bwd(const double *Q, const double *K, const double *V, const double *dO,
                const int32_t *row_ids, const int32_t *col_ids, int B, int H, int N, int d, int P,
-               const uint8_t *head_view, double scale, int radius, double *dQ, double *dK, double *dV) {
+               const uint8_t *head_view, double scale, int radius, int G, double *dQ, double *dK, double *dV) {
     uint8_t *M[3];
     for (int v = 0; v < 3; ++v) M[v] = (uint8_t *)malloc((size_t)N * N);
     double *LSE = (double *)malloc(sizeof(double) * (size_t)H * N);
@@ -216,7 +225,7 @@ int oracle_bwd(const double *Q, const double *K, const double *V, const double *
     if (!M[0] || !M[1] || !M[2] || !LSE || !D) return -1;
     for (int b = 0; b < B; ++b) {
         for (int view = 0; view < 3; ++view)
-            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, M[view]);
+            mask_of_pattern(row_ids + (size_t)b * N, col_ids + (size_t)b * N, N, P, view, radius, G, M[view]);
         /* pass 1, one query row at a time: LSE_k, D_k, dQ_k */
 #pragma omp parallel
         {

@@ -41,13 +41,19 @@ def num_threads() -> int:
     return int(_load().oracle_num_threads())
 
 
-def mask(row_ids, col_ids, P, view, radius=0):
+def _g(P, global_len):
+    return int(P if global_len is None else global_len)
+
+
+def mask(row_ids, col_ids, P, view, radius=0, global_len=None):
     """Explicit attention pattern of Section 3 for one example: uint8 [N, N], M[k, j] = j in A_k.
-    radius > 0: the bucketed pattern of Section 3.1 (buckets of `radius` positions of the view order)."""
+    radius > 0: the bucketed pattern of Section 3.1 (buckets of `radius` positions of the view order
+    behind a global section of global_len >= P positions; default: the prefix)."""
     r, c = _i32(row_ids).reshape(-1), _i32(col_ids).reshape(-1)
     N = r.shape[0]
     M = np.empty((N, N), dtype=np.uint8)
-    _load().oracle_mask_bucketed(_p(r), _p(c), C.c_int(N), C.c_int(P), C.c_int(view), C.c_int(radius), _p(M))
+    _load().oracle_mask_bucketed(_p(r), _p(c), C.c_int(N), C.c_int(P), C.c_int(view), C.c_int(radius),
+                                 C.c_int(_g(P, global_len)), _p(M))
     return M
 
 
@@ -73,16 +79,16 @@ def cell_mean(logits, row_ids, col_ids, P, max_row_id, max_col_id):
     return mean, cnt
 
 
-def useful_pairs(row_ids, col_ids, P, head_view, radius=0):
+def useful_pairs(row_ids, col_ids, P, head_view, radius=0, global_len=None):
     r, c, hv = _i32(row_ids), _i32(col_ids), _u8(head_view)
     B, N = r.shape
     out = np.zeros((B, hv.shape[0]), dtype=np.int64)
     _load().oracle_useful_pairs(_p(r), _p(c), C.c_int(B), C.c_int(hv.shape[0]), C.c_int(N),
-                                C.c_int(P), _p(hv), C.c_int(radius), _p(out))
+                                C.c_int(P), _p(hv), C.c_int(radius), C.c_int(_g(P, global_len)), _p(out))
     return out
 
 
-def fwd(Q, K, V, row_ids, col_ids, P, head_view, scale, radius=0):
+def fwd(Q, K, V, row_ids, col_ids, P, head_view, scale, radius=0, global_len=None):
     """Masked softmax attention (Section 3 head formula).  Returns O [B,H,N,d], LSE [B,H,N] (f64)."""
     Q, K, V = _f64(Q), _f64(K), _f64(V)
     r, c, hv = _i32(row_ids), _i32(col_ids), _u8(head_view)
@@ -92,12 +98,13 @@ def fwd(Q, K, V, row_ids, col_ids, P, head_view, scale, radius=0):
     O = np.empty_like(Q)
     LSE = np.empty((B, H, N), dtype=np.float64)
     rc = _load().oracle_fwd(_p(Q), _p(K), _p(V), _p(r), _p(c), C.c_int(B), C.c_int(H), C.c_int(N),
-                            C.c_int(d), C.c_int(P), _p(hv), C.c_double(scale), C.c_int(radius), _p(O), _p(LSE))
+                            C.c_int(d), C.c_int(P), _p(hv), C.c_double(scale), C.c_int(radius),
+                            C.c_int(_g(P, global_len)), _p(O), _p(LSE))
     assert rc == 0
     return O, LSE
 
 
-def bwd(Q, K, V, dO, row_ids, col_ids, P, head_view, scale, radius=0):
+def bwd(Q, K, V, dO, row_ids, col_ids, P, head_view, scale, radius=0, global_len=None):
     """Analytic backward of `fwd`.  Returns dQ, dK, dV (f64)."""
     Q, K, V, dO = _f64(Q), _f64(K), _f64(V), _f64(dO)
     r, c, hv = _i32(row_ids), _i32(col_ids), _u8(head_view)
@@ -107,7 +114,7 @@ def bwd(Q, K, V, dO, row_ids, col_ids, P, head_view, scale, radius=0):
     dQ, dK, dV = np.empty_like(Q), np.empty_like(Q), np.empty_like(Q)
     rc = _load().oracle_bwd(_p(Q), _p(K), _p(V), _p(dO), _p(r), _p(c), C.c_int(B), C.c_int(H),
                             C.c_int(N), C.c_int(d), C.c_int(P), _p(hv), C.c_double(scale), C.c_int(radius),
-                            _p(dQ), _p(dK), _p(dV))
+                            C.c_int(_g(P, global_len)), _p(dQ), _p(dK), _p(dV))
     assert rc == 0
     return dQ, dK, dV
 

@@ -11,23 +11,48 @@ from tests.test_oracle_pins import brute_fwd, brute_sets, rand_qkv, small_table
 from workloads import tables
 
 
-def brute_bucketed_sets(row_ids, col_ids, P, view, R):
+def brute_bucketed_sets(row_ids, col_ids, P, view, R, G=None):
     """Token by token, from the text: order the tokens (prefix first, then by row / column number,
-    ties by position, padding last), cut what follows the prefix into buckets of R, and keep of the
-    exact set A_k the prefix and the tokens whose bucket is the token's own or next to it."""
+    ties by position, padding last); the first G positions of that order (default: the prefix) are
+    global -- they see everything and everything sees them; what follows is cut into buckets of R,
+    and such a token keeps of the exact set A_k the global tokens and the tokens whose bucket is its
+    own or next to it."""
     ids = row_ids if view == 0 else col_ids
     N = len(ids)
+    G = P if G is None else max(G, P)
     exact = brute_sets(row_ids, col_ids, P, view)
     order = sorted(range(N), key=lambda k: ((0, 0) if k < P else ((1, ids[k]) if ids[k] >= 0 else (2, 0)), k))
     pos = {k: t for t, k in enumerate(order)}
-    bucket = {k: (pos[k] - P) // R for k in range(P, N)}
+    valid = [j for j in range(N) if ids[j] >= 0]
+    glob = set(j for j in valid if pos[j] < G)
+    bucket = {k: (pos[k] - G) // R for k in valid if pos[k] >= G}
     sets = []
     for k in range(N):
-        if k < P or ids[k] < 0:
-            sets.append(exact[k])
+        if ids[k] < 0:
+            sets.append(set())
+        elif k in glob:
+            sets.append(set(valid))
         else:
-            sets.append(set(j for j in exact[k] if j < P or abs(bucket[j] - bucket[k]) <= 1))
+            sets.append(glob | set(j for j in exact[k] if j not in glob and abs(bucket[j] - bucket[k]) <= 1))
     return sets
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+@pytest.mark.parametrize("R,G", [(2, 5), (3, 7), (1, 4), (4, 30)])
+def test_bucketed_mask_with_a_global_section_longer_than_the_prefix(seed, R, G):
+    # Section 3.1: the first G tokens of a head's order attend to and from everything, G >= |Q|; with
+    # G > |Q| the table tokens that come first in the head's order are global too
+    rows, cols, n = small_table(seed, P=3, n_rows=3, n_cols=3, max_len=3, pad=2)
+    for view in (0, 1):
+        M = oracle.mask(rows[0], cols[0], 3, view, radius=R, global_len=G)
+        sets = brute_bucketed_sets(list(rows[0]), list(cols[0]), 3, view, R, G)
+        for k in range(n):
+            assert set(np.nonzero(M[k])[0].tolist()) == sets[k], (view, k)
+        assert np.array_equal(M, M.T)
+        assert np.all(oracle.mask(rows[0], cols[0], 3, view, radius=R) <= M) or G > 3   # more global tokens, other buckets
+    # G = |Q| is the plain bucketed pattern; G below |Q| reads as |Q|
+    assert np.array_equal(oracle.mask(rows[0], cols[0], 3, 0, radius=R, global_len=3), oracle.mask(rows[0], cols[0], 3, 0, radius=R))
+    assert np.array_equal(oracle.mask(rows[0], cols[0], 3, 0, radius=R, global_len=1), oracle.mask(rows[0], cols[0], 3, 0, radius=R))
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2])
