@@ -60,6 +60,19 @@ enum { MATE_VIEW_ROW = 0, MATE_VIEW_COL = 1 }; /* entries of head_view          
  *   TCGEN05  tensor-core kernels or MATE_ERR_UNSUPPORTED */
 enum { MATE_IMPL_AUTO = 0, MATE_IMPL_SIMT = 1, MATE_IMPL_TCGEN05 = 2 };
 
+/* further flag bits (or-ed to the implementation choice):
+ *   VIEW_ORDER   (mate_attn_fwd only) Q, K, V are laid out, head by head, in that head's own order
+ *                (row b, h, t of a tensor holds the token at position t of the order mate_plan computed
+ *                for the head's view), and O and LSE are returned in the same order: what a producer
+ *                that writes its projections through the plan's order provides (Section 3.1: the
+ *                reordering can be folded into the neighbouring steps).  No gather, no scatter; the
+ *                tensor-core kernel then fetches every full tile with bulk tensor copies.  Not for
+ *                mate_plan_sat plans and not for mate_attn_bwd (MATE_ERR_UNSUPPORTED).
+ *   GATHER_ONLY  the tensor-core forward fetches every tile with row-by-row gathers, also those that
+ *                are contiguous in the tensors (which otherwise come in by bulk tensor copies): for
+ *                comparing the two load paths. */
+enum { MATE_FLAG_VIEW_ORDER = 4, MATE_FLAG_GATHER_ONLY = 8 };
+
 const char *mate_status_string(int status);
 
 /* Pre-computes, for both views, the per-head token order of Section 3.1 (Figure 2): a stable
@@ -101,6 +114,19 @@ int mate_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int 
 int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, int N, int prefix_len,
                        const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
                        void *stream, mate_plan_t **out);
+
+/* The bucketed form with a global section that may be longer than the prefix (Section 3.1: the first
+ * G tokens of a head's order attend to and from everything, with G at least the length of the
+ * question; Appendix A.2 uses G = 116, R = 42): the first global_len[b] positions of each head's
+ * own order -- the prefix and, beyond it, the table tokens that come first in that order -- see
+ * every non-padding position and are seen by all of them; the positions behind are cut into
+ * buckets of `radius`, counted from global_len[b], and attend the global section plus, of their own
+ * row / column, their own bucket and the two adjacent ones.  prefix_len and global_len are HOST
+ * int32 [B] arrays with prefix_len[b] <= global_len[b] <= N; radius > 0.  global_len = prefix_len
+ * is mate_plan_varlen.  All other arguments, ownership and errors as for mate_plan. */
+int mate_plan_bucketed_global(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
+                              const int32_t *global_len, const uint8_t *head_view, int H, int max_row_id,
+                              int max_col_id, int radius, void *stream, mate_plan_t **out);
 
 /* The same with one prefix length per example (the paper's inputs are a question or a passage of
  * varying length followed by the table, Section 3 and Section 5; its formula takes the set Q per
@@ -145,6 +171,14 @@ int mate_plan_useful_pairs(const mate_plan_t *plan, int64_t *pairs);
  * bounded wait since the last call (its outputs are then undefined), MATE_ERR_CUDA if the stream
  * reports an error, else MATE_OK. */
 int mate_plan_status(const mate_plan_t *plan, void *stream);
+
+/* Test hook (the paper has no counterpart): launches a one-thread kernel that waits, with the
+ * bounded helper the attention kernels use and a limit of a few tries (a few microseconds each), on a
+ * barrier that nothing arrives on; the wait gives up, the kernel raises the plan's time-out word as
+ * the attention kernels would, and returns.  The next mate_plan_status on the plan then reports
+ * MATE_ERR_TIMEOUT once, and the plan stays usable.  Lets the time-out path be exercised without
+ * making any real kernel wait in vain. */
+int mate_debug_expire_wait(const mate_plan_t *plan, void *stream);
 
 int mate_plan_destroy(mate_plan_t *plan);
 

@@ -9,6 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libmate.so")
 
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+FLAG_VIEW_ORDER, FLAG_GATHER_ONLY = 4, 8   # or-ed to the implementation choice (see mate.h)
 VIEW_ROW, VIEW_COL = 0, 1
 _BF16, _F32 = 0, 1
 
@@ -44,6 +45,8 @@ def _load():
     lib.mate_plan_bucketed.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_varlen.restype = i32
     lib.mate_plan_varlen.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
+    lib.mate_plan_bucketed_global.restype = i32
+    lib.mate_plan_bucketed_global.argtypes = [vp, vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_sat.restype = i32
     lib.mate_plan_sat.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_get.restype = i32
@@ -52,6 +55,8 @@ def _load():
     lib.mate_plan_useful_pairs.argtypes = [vp, vp]
     lib.mate_plan_status.restype = i32
     lib.mate_plan_status.argtypes = [vp, vp]
+    lib.mate_debug_expire_wait.restype = i32
+    lib.mate_debug_expire_wait.argtypes = [vp, vp]
     lib.mate_plan_destroy.restype = i32
     lib.mate_plan_destroy.argtypes = [vp]
     lib.mate_attn_workspace_bytes.restype = i32
@@ -125,6 +130,10 @@ class Plan:
     def status(self):
         _check(_load().mate_plan_status(self._h, _stream()), "mate_plan_status")
 
+    def debug_expire_wait(self):
+        """Test hook: makes a bounded device wait give up (see mate_debug_expire_wait in mate.h)."""
+        _check(_load().mate_debug_expire_wait(self._h, _stream()), "mate_debug_expire_wait")
+
     def destroy(self):
         if self._h is not None:
             _load().mate_plan_destroy(self._h)
@@ -178,6 +187,27 @@ def mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id=None, max_col_
         else:
             _check(lib.mate_plan(*common, int(prefix_len), *tail, _stream(), C.byref(handle)), "mate_plan")
     return Plan(handle, B, N, prefix_len, int(hv.shape[0]), int(max_row_id), int(max_col_id), row_ids.device)
+
+
+def mate_plan_bucketed_global(row_ids, col_ids, prefix_lens, global_lens, head_view, radius, max_row_id=None,
+                              max_col_id=None) -> Plan:
+    """Bucketed plan whose global section (global_lens[b] >= prefix_lens[b] positions of every head's own order)
+    may reach beyond the prefix (see mate_plan_bucketed_global in mate.h).  Scalars are taken for every example."""
+    B, N = row_ids.shape
+    pf = np.ascontiguousarray(np.broadcast_to(np.asarray(prefix_lens, dtype=np.int32), (B,)))
+    gl = np.ascontiguousarray(np.broadcast_to(np.asarray(global_lens, dtype=np.int32), (B,)))
+    hv = np.ascontiguousarray(np.asarray(head_view, dtype=np.uint8))
+    if max_row_id is None:
+        max_row_id = max(int(row_ids.max().item()), 0)
+    if max_col_id is None:
+        max_col_id = max(int(col_ids.max().item()), 0)
+    handle = C.c_void_p()
+    with torch.cuda.device(row_ids.device):
+        _check(_load().mate_plan_bucketed_global(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, N, pf.ctypes.data,
+                                                 gl.ctypes.data, hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
+                                                 int(max_col_id), int(radius), _stream(), C.byref(handle)),
+               "mate_plan_bucketed_global")
+    return Plan(handle, B, N, pf.tolist(), int(hv.shape[0]), int(max_row_id), int(max_col_id), row_ids.device)
 
 
 def mate_plan_sat(row_ids, col_ids, prefix_len, n_heads, max_row_id=None, max_col_id=None) -> Plan:
@@ -260,7 +290,7 @@ def mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale=None, impl=IMPL_AUTO, workspa
     return dQ, dK, dV
 
 
-def mate_cell_mean(plan, logits, col_ids, want_count=True):
+def mate_cell_mean(plan, logits, col_ids, want_count=True, out=None):
     """Mean of the token logits per table cell (see mate_cell_mean in mate.h).  logits: float32 [B, N];
     col_ids: the int32 [B, N] tensor the plan was made from.  Returns (mean, count) of shape
     [B, max_row_id + 1, max_col_id + 1] (count is None when not wanted)."""
@@ -269,8 +299,12 @@ def mate_cell_mean(plan, logits, col_ids, want_count=True):
     if col_ids.dtype != torch.int32 or tuple(col_ids.shape) != (plan.B, plan.N):
         raise ValueError("col_ids must be the int32 [B, N] tensor given to mate_plan")
     shape = (plan.B, plan.max_id[0] + 1, plan.max_id[1] + 1)
-    mean = torch.empty(shape, dtype=torch.float32, device=logits.device)
-    count = torch.empty(shape, dtype=torch.int32, device=logits.device) if want_count else None
+    if out is not None:  # (mean, count) tensors of an earlier call, written in place
+        mean, count = out
+        want_count = count is not None
+    else:
+        mean = torch.empty(shape, dtype=torch.float32, device=logits.device)
+        count = torch.empty(shape, dtype=torch.int32, device=logits.device) if want_count else None
     with torch.cuda.device(logits.device):
         _check(_load().mate_cell_mean(plan._h, _dev(logits, "logits"), _dev(col_ids, "col_ids"), _dev(mean, "mean"),
                                       _dev(count, "count") if want_count else None, _stream()), "mate_cell_mean")

@@ -42,9 +42,11 @@ void carve(mate_plan_t *pl, char *base, size_t *total) {
         vp.seg_hi = c.take<int32_t>(BN);
         vp.seg_off = c.take<int32_t>(S);
         vp.cursor = c.take<int32_t>(S);
+        vp.ident = c.take<int32_t>(pl->B);
     }
     pl->n_valid_dev = c.take<int32_t>(pl->B);
     pl->prefix_dev = c.take<int32_t>(pl->B);
+    pl->global_dev = c.take<int32_t>(pl->B);
     pl->status_dev = c.take<int32_t>(4);
     pl->head_view_dev = c.take<uint8_t>(pl->H);
     *total = align_up(c.off, 256);
@@ -69,7 +71,7 @@ struct UnitCost {
 // three adjacent buckets when the plan is bucketed.  The same arithmetic as step 4 of the plan kernel.
 struct RowBounds {
     const int32_t *so;
-    int S, P, radius;
+    int S, P, radius;  // P: length of the global block (bucket origin; no range reaches in front of it)
     int mode = mate::kBoundsOwn, group = 1;
     int seg_of(int t) const { return (int)(std::upper_bound(so, so + S, t) - so) - 1; }
     int lo(int t) const {
@@ -77,18 +79,20 @@ struct RowBounds {
         int l = so[id];
         if (mode == mate::kBoundsBefore) l = so[id / group * group];
         if (mode == mate::kBoundsAfter) l = so[id + 1];
-        if (radius <= 0) return l;
+        if (radius <= 0) return std::max(l, P);
         const int64_t bk = (t - P) / radius;
-        return (int)std::max<int64_t>(l, P + (bk - 1) * radius);
+        return (int)std::max<int64_t>(std::max(l, P), P + (bk - 1) * radius);
     }
     int hi(int t) const {
         const int id = seg_of(t);
         int h = so[id + 1];
         if (mode == mate::kBoundsBefore) h = so[id];
         if (mode == mate::kBoundsAfter) h = so[std::min((id / group + 1) * group, S - 1)];
-        if (radius <= 0) return h;
-        const int64_t bk = (t - P) / radius;
-        return (int)std::min<int64_t>(h, P + (bk + 2) * radius);
+        if (radius > 0) {
+            const int64_t bk = (t - P) / radius;
+            h = (int)std::min<int64_t>(h, P + (bk + 2) * radius);
+        }
+        return std::max(h, lo(t));
     }
 };
 
@@ -126,7 +130,7 @@ void make_units(mate_plan_t *pl, const std::vector<std::vector<int32_t>> &seg_of
         for (int b = 0; b < pl->B; ++b) {
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
             const int nv = pl->n_valid[b];
-            const int P = pl->prefix[b];
+            const int P = std::min(pl->global[b], nv);  // rows and keys in front of it are global
             const RowBounds rb{so, S, P, pl->radius, pl->bounds_mode, pl->group};
             std::vector<UnitCost> proto;  // units of one (example, view); copied per head below
             for (int q0 = 0; q0 < P; q0 += mate::kUnitRows) {  // prefix rows: every valid key
@@ -289,13 +293,24 @@ int mate_plan_bucketed(const int32_t *row_ids, const int32_t *col_ids, int B, in
 }
 
 static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
-                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius, int bounds_mode,
-                      int group, void *stream, mate_plan_t **out);
+                      const int32_t *global_len, const uint8_t *head_view, int H, int max_row_id, int max_col_id,
+                      int radius, int bounds_mode, int group, void *stream, mate_plan_t **out);
 
 int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
                      void *stream, mate_plan_t **out) {
-    return build_plan(row_ids, col_ids, B, N, prefix_len, head_view, H, max_row_id, max_col_id, radius,
+    return build_plan(row_ids, col_ids, B, N, prefix_len, nullptr, head_view, H, max_row_id, max_col_id, radius,
+                      mate::kBoundsOwn, 1, stream, out);
+}
+
+int mate_plan_bucketed_global(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
+                              const int32_t *global_len, const uint8_t *head_view, int H, int max_row_id,
+                              int max_col_id, int radius, void *stream, mate_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!global_len || !prefix_len || B <= 0 || radius <= 0) return MATE_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b)
+        if (global_len[b] < prefix_len[b] || global_len[b] > N) return MATE_ERR_INVALID_ARG;
+    return build_plan(row_ids, col_ids, B, N, prefix_len, global_len, head_view, H, max_row_id, max_col_id, radius,
                       mate::kBoundsOwn, 1, stream, out);
 }
 
@@ -314,7 +329,7 @@ int mate_plan_sat(const int32_t *row_ids, const int32_t *col_ids, int B, int N, 
     const std::vector<int32_t> prefix((size_t)B, prefix_len), zero((size_t)B, 0);
     const std::vector<uint8_t> rows_only((size_t)H, 0), cols_only((size_t)H, 1);
     mate_plan_t *pl = nullptr;
-    int rc = build_plan(row_ids, col_ids, B, N, prefix.data(), rows_only.data(), H, max_row_id, max_col_id, 0,
+    int rc = build_plan(row_ids, col_ids, B, N, prefix.data(), nullptr, rows_only.data(), H, max_row_id, max_col_id, 0,
                         mate::kBoundsOwn, 1, stream, &pl);
     if (rc != MATE_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
@@ -327,7 +342,7 @@ int mate_plan_sat(const int32_t *row_ids, const int32_t *col_ids, int B, int N, 
         return MATE_ERR_NOMEM;
     }
     for (int s = 0; s < 2 && rc == MATE_OK; ++s)
-        rc = build_plan(pl->pair_ids_dev, pl->pair_ids_dev, B, N, zero.data(), cols_only.data(), H, max_pair, max_pair, 0,
+        rc = build_plan(pl->pair_ids_dev, pl->pair_ids_dev, B, N, zero.data(), nullptr, cols_only.data(), H, max_pair, max_pair, 0,
                         s == 0 ? mate::kBoundsBefore : mate::kBoundsAfter, n_row_ids, stream, &pl->sub[s]);
     if (rc != MATE_OK) {
         mate_plan_destroy(pl);
@@ -338,8 +353,8 @@ int mate_plan_sat(const int32_t *row_ids, const int32_t *col_ids, int B, int N, 
 }
 
 static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
-                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius, int bounds_mode,
-                      int group, void *stream, mate_plan_t **out) {
+                      const int32_t *global_len, const uint8_t *head_view, int H, int max_row_id, int max_col_id,
+                      int radius, int bounds_mode, int group, void *stream, mate_plan_t **out) {
     if (out) *out = nullptr;
     if (radius < 0) return MATE_ERR_INVALID_ARG;
     if (!row_ids || !col_ids || !head_view || !out || !prefix_len) return MATE_ERR_INVALID_ARG;
@@ -358,6 +373,8 @@ static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int
     pl->B = B;
     pl->N = N;
     pl->prefix.assign(prefix_len, prefix_len + B);
+    if (global_len) pl->global.assign(global_len, global_len + B);
+    else pl->global = pl->prefix;
     pl->H = H;
     pl->radius = radius;
     pl->bounds_mode = bounds_mode;
@@ -394,7 +411,9 @@ static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int
                                st) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(pl->prefix_dev, pl->prefix.data(), B * sizeof(int32_t), cudaMemcpyHostToDevice,
                                st) == cudaSuccess;
-    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, pl->prefix_dev, radius, bounds_mode, pl->group, pl->view[0], pl->view[1],
+    ok = ok && cudaMemcpyAsync(pl->global_dev, pl->global.data(), B * sizeof(int32_t), cudaMemcpyHostToDevice,
+                               st) == cudaSuccess;
+    ok = ok && mate::launch_plan_kernels(row_ids, col_ids, B, N, pl->prefix_dev, pl->global_dev, radius, bounds_mode, pl->group, pl->view[0], pl->view[1],
                                          pl->n_valid_dev, pl->status_dev, st) == cudaSuccess;
     for (int v = 0; v < 2 && ok; ++v) {
         seg_off_host[v].resize((size_t)B * (pl->view[v].max_id + 2));
@@ -421,9 +440,9 @@ static int build_plan(const int32_t *row_ids, const int32_t *col_ids, int B, int
         const int S = pl->view[v].max_id + 2;
         for (int b = 0; b < B; ++b) {
             const int32_t *so = seg_off_host[v].data() + (size_t)b * S;
-            const int P = pl->prefix[b];
+            const int P = std::min(pl->global[b], pl->n_valid[b]);
             int64_t c = (int64_t)P * pl->n_valid[b];
-            if (radius > 0 || pl->bounds_mode != mate::kBoundsOwn) {
+            if (radius > 0 || pl->bounds_mode != mate::kBoundsOwn || P != pl->prefix[b]) {
                 const RowBounds rb{so, S, P, radius, pl->bounds_mode, pl->group};
                 for (int t = P; t < pl->n_valid[b]; ++t) c += P + rb.hi(t) - rb.lo(t);
             } else {
@@ -524,7 +543,7 @@ static int check_common(const mate_plan_t *plan, int d, int dtype, unsigned flag
     if (dtype != MATE_BF16 && dtype != MATE_F32) return MATE_ERR_UNSUPPORTED;
     if (d <= 0 || d % 8 != 0 || d > 128) return MATE_ERR_UNSUPPORTED;
     const unsigned impl = flags & 3u;
-    if (impl == 3u) return MATE_ERR_INVALID_ARG;
+    if (impl == 3u || (flags & ~(3u | MATE_FLAG_VIEW_ORDER | MATE_FLAG_GATHER_ONLY))) return MATE_ERR_INVALID_ARG;
     const bool tc_ok = mate::tc_supported(d, dtype);
     if (impl == MATE_IMPL_TCGEN05 && !tc_ok) return MATE_ERR_UNSUPPORTED;
     *use_tc = (impl == MATE_IMPL_TCGEN05) || (impl == MATE_IMPL_AUTO && tc_ok);
@@ -562,9 +581,9 @@ int mate_attn_workspace_bytes(const mate_plan_t *plan, int d, int dtype, unsigne
 }
 
 static int fwd_pass(const mate_plan_t *plan, bool use_tc, const void *Q, const void *K, const void *V, int d, int dtype,
-                    float scale, void *O, float *LSE, void *ws, cudaStream_t st) {
-    if (use_tc) return mate::tc_fwd(plan, Q, K, V, scale, O, LSE, ws, st);
-    return mate::simt_fwd(plan, Q, K, V, d, dtype, scale, O, LSE, st);
+                    float scale, void *O, float *LSE, void *ws, unsigned flags, cudaStream_t st) {
+    if (use_tc) return mate::tc_fwd(plan, Q, K, V, scale, O, LSE, ws, flags, st);
+    return mate::simt_fwd(plan, Q, K, V, d, dtype, scale, O, LSE, flags, st);
 }
 
 int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d,
@@ -587,7 +606,8 @@ int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     mate_attn_workspace_bytes(plan, d, dtype, use_tc ? MATE_IMPL_TCGEN05 : MATE_IMPL_SIMT, &need, nullptr);
     if (need > 0 && (!workspace || workspace_bytes < need)) return MATE_ERR_WORKSPACE;
     if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MATE_ERR_ALIGNMENT;
-    rc = fwd_pass(plan, use_tc, Q, K, V, d, dtype, scale, O, LSE, workspace, st);
+    if ((flags & MATE_FLAG_VIEW_ORDER) && plan->sub[0]) return MATE_ERR_UNSUPPORTED;  // the passes use different orders
+    rc = fwd_pass(plan, use_tc, Q, K, V, d, dtype, scale, O, LSE, workspace, flags, st);
     if (rc != MATE_OK || !plan->sub[0]) return rc;
     // row-or-column pattern: the two passes over the rest of the column, then the merge
     const size_t rows = (size_t)plan->B * plan->H * plan->N;
@@ -599,7 +619,7 @@ int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const v
         Os[s] = w;
         Ls[s] = (float *)(w + o_bytes);
         w += o_bytes + l_bytes;
-        rc = fwd_pass(plan->sub[s], use_tc, Q, K, V, d, dtype, scale, Os[s], Ls[s], workspace, st);
+        rc = fwd_pass(plan->sub[s], use_tc, Q, K, V, d, dtype, scale, Os[s], Ls[s], workspace, flags, st);
         if (rc != MATE_OK) return rc;
     }
     return mate::launch_merge_passes(O, LSE, Os[0], Ls[0], Os[1], Ls[1], rows, d, dtype, st) == cudaSuccess ? MATE_OK
@@ -622,6 +642,7 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     if (rc != MATE_OK) return rc;
     if ((rc = check_device(plan)) != MATE_OK) return rc;
     if (!Q || !K || !V || !O || !LSE || !dO || !dQ || !dK || !dV) return MATE_ERR_INVALID_ARG;
+    if (flags & MATE_FLAG_VIEW_ORDER) return MATE_ERR_UNSUPPORTED;  // forward only
     const void *ptrs[] = {Q, K, V, O, LSE, dO, dQ, dK, dV};
     for (const void *p : ptrs)
         if (!aligned16(p)) return MATE_ERR_ALIGNMENT;

@@ -22,6 +22,7 @@
 // they meet the segments of its rows, and inside a tile a warp evaluates only the 32-column chunks
 // that meet the segments of its 32 rows.  The scatter back to the original token order is fused
 // into the epilogue (each thread stores its 128-byte row at the row's original position).
+#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "mate_internal.h"
@@ -81,6 +82,10 @@ constexpr int kSchedReaders = kSoftmaxWarps + kMmaWarps + kLoadWarps;
 static_assert(kStages <= 5, "barrier slots");
 
 struct Params {
+    // 2-D tensor maps over Q, K, V seen as [B H N rows, 64 columns]: boxes of 128 rows, 128-byte swizzle
+    CUtensorMap tmQ, tmK, tmV;
+    int use_tma;     // 0: every tile is gathered row by row
+    int view_order;  // 1: Q, K, V, O and LSE are laid out in each head's own order (no gather, no scatter)
     const __nv_bfloat16 *Q, *K, *V;
     __nv_bfloat16 *O;
     float *LSE;
@@ -154,7 +159,8 @@ __device__ __forceinline__ void load_indices(int (&idx)[kPasses], const int32_t 
 #pragma unroll
     for (int i = 0; i < kPasses; ++i) {
         const int rr = (ltid >> 3) + kRowsPerPass * i;
-        idx[i] = rr < n_rows ? __ldg(perm + row0 + min(rr, clamp)) : -1;
+        const int t = row0 + min(rr, clamp);
+        idx[i] = rr < n_rows ? (perm ? __ldg(perm + t) : t) : -1;  // no order given: the tensors are in view order
     }
 }
 __device__ __forceinline__ void copy_rows(uint32_t s_tile, const __nv_bfloat16 *src_bh,
@@ -212,7 +218,7 @@ __device__ __forceinline__ float sum_f32x2(uint64_t a, uint64_t b) {
     return (a0 + a1) + (b0 + b1);
 }
 
-__global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
+__global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_constant__ Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -310,7 +316,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
             const bool row_valid = r < rows_h;
             const int t_row = un.q0 + h * kTile + min(r, rows_h - 1);  // rows past the end shadow the last one
-            const int orig = perm[t_row];
+            const int orig = p.view_order ? t_row : perm[t_row];
             const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
             const int h_lo = h ? un.lo[1] : un.lo[0], h_hi = h ? un.hi[1] : un.hi[0];  // segments of this half's rows
 
@@ -836,37 +842,73 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
             const int nA = n_tiles_a(un), nB = n_tiles_b(un), n_tiles = nA + nB;
             if (n_tiles == 0) continue;
             const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
-            const int32_t *perm = vp.perm + (size_t)un.b * p.N;
+            const int32_t *perm = p.view_order ? nullptr : vp.perm + (size_t)un.b * p.N;
             const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
             const __nv_bfloat16 *Qbh = p.Q + bh * 64, *Kbh = p.K + bh * 64, *Vbh = p.V + bh * 64;
+            // Rows of the order that sit in place in the tensors ([0, ident)): a full tile inside that
+            // range is one contiguous [128, 64] box and comes in by one bulk tensor copy per matrix
+            // (issued by one thread, completing on the tile's barrier by byte count) instead of 2 x 1024
+            // gathered 16-byte copies.  That is the prefix block of every unit and, for a row-major
+            // table, every tile of the row view.
+            const int ident = !p.use_tma ? 0 : p.view_order ? p.N : __ldg(vp.ident + un.b);
 
             const int qb = unit_cnt & 1;
             if (!(alive = wait_free(bars + 8 * (kBarQEmpty + qb), ((unit_cnt >> 1) & 1) ^ 1))) break;
-            for (int h = 0; h < 2; ++h) {
-                const int rows_h = rows_of_half(un, h);
-                if (rows_h > 0) {
-                    int idx[kPasses];
-                    load_indices(idx, perm, un.q0 + h * kTile, kTile, rows_h - 1, ltid);
-                    copy_rows(base + kOffQ + (qb * 2 + h) * kTileBytes, Qbh, idx, ltid);
+            {
+                const uint32_t bar_q = bars + 8 * (kBarQFull + qb);
+                bool gathered = false;
+                for (int h = 0; h < 2; ++h) {
+                    const int rows_h = rows_of_half(un, h);
+                    if (rows_h == 0) continue;
+                    const int r0 = un.q0 + h * kTile;
+                    const uint32_t dst = base + kOffQ + (qb * 2 + h) * kTileBytes;
+                    if (rows_h == kTile && r0 + kTile <= ident) {
+                        if (ltid == 0) {
+                            mbar_expect_tx(bar_q, kTileBytes);
+                            tma_load_2d(dst, &p.tmQ, 0, (int)bh + r0, bar_q);
+                        }
+                    } else {
+                        int idx[kPasses];
+                        load_indices(idx, perm, r0, kTile, rows_h - 1, ltid);
+                        copy_rows(dst, Qbh, idx, ltid);
+                        gathered = true;
+                    }
+                }
+                if (gathered) {
+                    commit_and_signal(bar_q);
+                } else {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_q);
                 }
             }
-            commit_and_signal(bars + 8 * (kBarQFull + qb));
             ++unit_cnt;
 
             for (int i = 0; i < n_tiles; ++i) {
                 const TileInfo t = tile_info(un, i, nA);
                 const int stage = kv_cnt % kStages;
+                const bool bulk = t.w == kTile && t.k0 + kTile <= ident;
                 int idx[kPasses];
-                load_indices(idx, perm, t.k0, (t.w + 15) & ~15, t.w - 1, ltid);
+                if (!bulk) load_indices(idx, perm, t.k0, (t.w + 15) & ~15, t.w - 1, ltid);
                 if (!(alive = wait_free(bars + 8 * (kBarKVEmpty + stage), ((kv_cnt / kStages) & 1) ^ 1))) break;
                 const uint32_t sK = base + kOffKV + stage * 2 * kTileBytes;
+                const uint32_t bar_kv = bars + 8 * (kBarKVFull + stage);
                 TR_T0(t_cp);
-                copy_rows(sK, Kbh, idx, ltid);
-                copy_rows(sK + kTileBytes, Vbh, idx, ltid);
-                TR_ADD(2, t_cp);
-                TR_T0(t_cs);
-                commit_and_signal(bars + 8 * (kBarKVFull + stage));
-                TR_ADD(3, t_cs);
+                if (bulk) {
+                    if (ltid == 0) {
+                        mbar_expect_tx(bar_kv, 2 * kTileBytes);
+                        tma_load_2d(sK, &p.tmK, 0, (int)bh + t.k0, bar_kv);
+                        tma_load_2d(sK + kTileBytes, &p.tmV, 0, (int)bh + t.k0, bar_kv);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_kv);
+                } else {
+                    copy_rows(sK, Kbh, idx, ltid);
+                    copy_rows(sK + kTileBytes, Vbh, idx, ltid);
+                    TR_ADD(2, t_cp);
+                    TR_T0(t_cs);
+                    commit_and_signal(bar_kv);
+                    TR_ADD(3, t_cs);
+                }
                 TR_INC(4);
                 ++kv_cnt;
             }
@@ -899,6 +941,36 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const Params p) {
 
 SmemAttrOnce g_smem_attr;
 
+// cuTensorMapEncodeTiled, taken from the driver through the runtime (the library does not link libcuda)
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(ptr);
+    }();
+    return fn;
+}
+
+// Map over a [rows, 64] bf16 matrix (row = 128 bytes): boxes of 128 rows, written to shared memory in
+// the 128-byte swizzle the tensor-core descriptors expect (16-byte chunk index XOR row & 7).
+bool make_row_map(CUtensorMap *map, const void *base, size_t rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {64, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {kRowBytes};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool tc_supported(int d, int dtype) { return d == 64 && dtype == MATE_BF16; }
@@ -908,11 +980,17 @@ int tc_fwd_ctas_per_sm() { return 1; }
 size_t tc_fwd_workspace(const mate_plan_t *plan, int) { return plan->fwd_ws_bytes; }
 
 int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, float scale, void *O,
-           float *LSE, void *workspace, cudaStream_t stream) {
+           float *LSE, void *workspace, unsigned flags, cudaStream_t stream) {
     if (!(scale > 0.f)) return MATE_ERR_UNSUPPORTED;  // the row max is taken before scaling (the caller falls back)
     if (plan->n_fwd_units == 0) return MATE_OK;
     if (g_smem_attr.ensure((const void *)tc_fwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
     Params p;
+    const size_t rows = (size_t)plan->B * plan->H * plan->N;
+    // bulk tensor copies for the tiles that are contiguous in the caller's tensors; without the driver
+    // entry point (or with MATE_FLAG_GATHER_ONLY) every tile is gathered row by row
+    p.use_tma = !(flags & MATE_FLAG_GATHER_ONLY) && rows < (size_t(1) << 31) && make_row_map(&p.tmQ, Q, rows) &&
+                make_row_map(&p.tmK, K, rows) && make_row_map(&p.tmV, V, rows);
+    p.view_order = (flags & MATE_FLAG_VIEW_ORDER) ? 1 : 0;
     p.Q = (const __nv_bfloat16 *)Q;
     p.K = (const __nv_bfloat16 *)K;
     p.V = (const __nv_bfloat16 *)V;

@@ -50,6 +50,7 @@ struct ViewPlan {
                                   //          plans: of the part of it within the adjacent buckets)
     int32_t *seg_hi = nullptr;    // [B, N]   one past the last key (prefix rows: n_valid; padding: 0)
     int32_t *cursor = nullptr;    // [B, max_id + 2] scratch of the counting sort
+    int32_t *ident = nullptr;     // [B]      number of leading view positions t with perm[t] = t
     int max_id = 0;
     int n_heads = 0;
 };
@@ -61,6 +62,11 @@ struct mate_plan_s {
     int device = 0;                      // ordinal of the device the plan's arrays live on
     std::vector<int32_t> prefix;         // |Q| per example (host copy)
     int32_t *prefix_dev = nullptr;       // [B]
+    // Length of the global block per example: the positions [0, G) of a head's order that see and are
+    // seen by everything.  G = |Q| except for a bucketed plan with a longer global section.  This, not
+    // |Q|, is what the attention kernels and the work-lists use; |Q| only decides the order.
+    std::vector<int32_t> global;
+    int32_t *global_dev = nullptr;       // [B]
     int radius = 0;                      // > 0: bucketed pattern (Section 3.1), buckets of this many positions
     int bounds_mode = 0, group = 1;      // key range of a table row (kBounds*), ids per group
     // row-or-column pattern (mate_plan_sat): this plan is the row pass; sub[0] / sub[1] are the passes
@@ -116,7 +122,8 @@ struct SmemAttrOnce {
 
 // plan kernels (mate_plan_kernels.cu)
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,
-                                const int32_t *prefix /* device [B] */, int radius, int bounds_mode, int group,
+                                const int32_t *prefix /* device [B] */, const int32_t *global_len /* device [B] */,
+                                int radius, int bounds_mode, int group,
                                 const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid, int32_t *status,
                                 cudaStream_t stream);
 cudaError_t launch_pair_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix,
@@ -129,7 +136,7 @@ cudaError_t launch_add3(void *a, const void *b, const void *c, size_t n, int dty
 
 // SIMT kernels (mate_simt.cu)
 int simt_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d, int dtype,
-             float scale, void *O, float *LSE, cudaStream_t stream);
+             float scale, void *O, float *LSE, unsigned flags, cudaStream_t stream);
 size_t simt_bwd_workspace(const mate_plan_t *plan);
 int simt_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, const void *O,
              const float *LSE, const void *dO, int d, int dtype, float scale, void *dQ, void *dK,
@@ -144,7 +151,7 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
            const float *LSE, const void *dO, float scale, void *dQ, void *dK, void *dV, void *workspace,
            cudaStream_t stream);
 int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, float scale, void *O,
-           float *LSE, void *workspace, cudaStream_t stream);
+           float *LSE, void *workspace, unsigned flags, cudaStream_t stream);
 
 }  // namespace mate
 

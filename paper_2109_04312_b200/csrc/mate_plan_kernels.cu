@@ -21,7 +21,8 @@ __device__ __forceinline__ int warp_inclusive_scan(int v, int lane) {
 
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, int N,
-            const int32_t *__restrict__ prefix, int radius, int bounds_mode, int group,
+            const int32_t *__restrict__ prefix, const int32_t *__restrict__ global_len, int radius, int bounds_mode,
+            int group,
             ViewPlan rowv, ViewPlan colv, int32_t *__restrict__ n_valid_out,
             int32_t *__restrict__ status) {
     __shared__ int32_t s_cursor[kSmemIds];
@@ -121,15 +122,31 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
     }
     __syncthreads();
 
+    // 3b. how many leading positions of the order are in place (perm[t] = t for every t below): rows
+    //     there are contiguous in the caller's tensors, which lets the attention kernels fetch whole
+    //     tiles with one bulk tensor copy instead of row-by-row gathers
+    {
+        __shared__ int s_ident;
+        if (tid == 0) s_ident = N;
+        __syncthreads();
+        int first_moved = N;
+        for (int t = tid; t < N; t += kPlanThreads)
+            if (perm[t] != t) first_moved = min(first_moved, t);
+        if (first_moved < N) atomicMin(&s_ident, first_moved);
+        __syncthreads();
+        if (tid == 0) vp.ident[b] = s_ident;
+    }
+
     // 4. per view position: its key range.  Normally its own segment; for the passes of the
     //    row-or-column pattern, whose ids are (column, row) pairs in groups of `group` ids per
     //    column, the segments of its group in front of / behind its own.  With a radius (the bucketed form of
     //    Section 3.1: the order behind the prefix is cut into buckets of `radius` positions and a
     //    token sees its own bucket and the two next to it) the range is clipped to those buckets.
     int32_t *seg_lo = vp.seg_lo + (size_t)b * N, *seg_hi = vp.seg_hi + (size_t)b * N;
+    const int G = global_len[b];  // the first G positions of the order see and are seen by everything (G >= P)
     for (int t = tid; t < N; t += kPlanThreads) {
         int lo = 0, hi = 0;
-        if (t < P) {
+        if (t < min(G, n_valid)) {
             hi = n_valid;
         } else if (t < n_valid) {
             int id = ids[perm[t]];
@@ -143,11 +160,13 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
                 hi = seg_off[min((id / group + 1) * group, vp.max_id + 1)];
             }
             if (radius > 0) {
-                const long long bk = (t - P) / radius;
-                const long long w0 = P + (bk - 1) * radius, w1 = P + (bk + 2) * radius;
+                const long long bk = (t - G) / radius;
+                const long long w0 = G + (bk - 1) * radius, w1 = G + (bk + 2) * radius;
                 lo = (int)max((long long)lo, w0);
                 hi = (int)min((long long)hi, w1);
             }
+            lo = max(lo, G);  // keys in front of G belong to the global block
+            hi = max(hi, lo);
         }
         seg_lo[t] = lo;
         seg_hi[t] = hi;
@@ -157,11 +176,12 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
 }  // namespace
 
 cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, int B, int N,
-                                const int32_t *prefix, int radius, int bounds_mode, int group, const ViewPlan &rowv,
-                                const ViewPlan &colv, int32_t *n_valid, int32_t *status, cudaStream_t stream) {
+                                const int32_t *prefix, const int32_t *global_len, int radius, int bounds_mode, int group,
+                                const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid, int32_t *status,
+                                cudaStream_t stream) {
     dim3 grid(B, 2);
-    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, prefix, radius, bounds_mode, max(group, 1), rowv,
-                                                   colv, n_valid, status);
+    plan_kernel<<<grid, kPlanThreads, 0, stream>>>(row_ids, col_ids, N, prefix, global_len, radius, bounds_mode,
+                                                   max(group, 1), rowv, colv, n_valid, status);
     return cudaGetLastError();
 }
 

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__restrict__ V,
                 T *__restrict__ O, float *__restrict__ LSE, ViewPlan rowv, ViewPlan colv,
                 const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
-                const int32_t *__restrict__ prefix, int d, float scale) {
+                const int32_t *__restrict__ prefix, int d, float scale, int view_order) {
     __shared__ float s_q[kWarpsPerBlock][kMaxD];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kWarpsPerBlock + warp;
@@ -83,7 +83,7 @@ simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
     if (t >= N) return;
     const RowCtx c = row_ctx(rowv, colv, head_view, n_valid, b, h, N);
     const size_t bh = ((size_t)b * H + h) * N;
-    const int k = c.perm[t];
+    const int k = view_order ? t : c.perm[t];  // view order: the tensors are laid out in the head's own order
     T *o_row = O + (bh + k) * d;
     if (t >= c.n_valid) {  // padding query row
         for (int e = lane; e < d; e += 32) from_f(o_row[e], 0.f);
@@ -97,14 +97,14 @@ simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
 #pragma unroll
     for (int i = 0; i < kAccPerLane; ++i) acc[i] = 0.f;
 
-    const int P = prefix[b];
+    const int P = min(prefix[b], c.n_valid);  // length of the global block (never reaches into the padding)
     const int lo = max(c.seg_lo[t], P), hi = c.seg_hi[t];
     for (int range = 0; range < 2; ++range) {
         const int j_begin = range ? lo : 0, j_end = range ? hi : P;
         for (int j0 = j_begin; j0 < j_end; j0 += 32) {
             const int j = j0 + lane;
             const bool on = j < j_end;
-            const int kj = on ? c.perm[j] : 0;
+            const int kj = on ? (view_order ? j : c.perm[j]) : 0;
             float s = on ? scale * dot_row(s_q[warp], K + (bh + kj) * d, d) : -INFINITY;
             const float m_new = fmaxf(m, warp_max(s));
             const float p = on ? expf(s - m_new) : 0.f;
@@ -197,7 +197,7 @@ simt_bwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
 #pragma unroll
     for (int i = 0; i < kAccPerLane; ++i) acc0[i] = acc1[i] = 0.f;
 
-    const int P = prefix[b];
+    const int P = min(prefix[b], c.n_valid);  // length of the global block (never reaches into the padding)
     const int lo = max(c.seg_lo[t], P), hi = c.seg_hi[t];
     for (int range = 0; range < 2; ++range) {
         const int j_begin = range ? lo : 0, j_end = range ? hi : P;
@@ -248,11 +248,11 @@ simt_bwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
 
 template <typename T>
 int simt_fwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *V, int d, float scale,
-               void *O, float *LSE, cudaStream_t st) {
+               void *O, float *LSE, int view_order, cudaStream_t st) {
     dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
     simt_fwd_kernel<T><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (T *)O, LSE, pl->view[0], pl->view[1],
-        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->prefix_dev, d, scale);
+        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale, view_order);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
@@ -267,20 +267,21 @@ int simt_bwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *
     dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
     simt_bwd_kernel<T, false><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
-        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->prefix_dev, d, scale);
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale);
     simt_bwd_kernel<T, true><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
-        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->prefix_dev, d, scale);
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale);
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
 }  // namespace
 
 int simt_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V, int d, int dtype,
-             float scale, void *O, float *LSE, cudaStream_t stream) {
+             float scale, void *O, float *LSE, unsigned flags, cudaStream_t stream) {
     if (d > kMaxD) return MATE_ERR_UNSUPPORTED;
-    return dtype == MATE_F32 ? simt_fwd_t<float>(plan, Q, K, V, d, scale, O, LSE, stream)
-                             : simt_fwd_t<__nv_bfloat16>(plan, Q, K, V, d, scale, O, LSE, stream);
+    const int vo = (flags & MATE_FLAG_VIEW_ORDER) ? 1 : 0;
+    return dtype == MATE_F32 ? simt_fwd_t<float>(plan, Q, K, V, d, scale, O, LSE, vo, stream)
+                             : simt_fwd_t<__nv_bfloat16>(plan, Q, K, V, d, scale, O, LSE, vo, stream);
 }
 
 size_t simt_bwd_workspace(const mate_plan_t *plan) {

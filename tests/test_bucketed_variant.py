@@ -146,3 +146,55 @@ def test_bucketed_forward_backward_parity(name, R, impl_idx):
     for nm, g, o in (("dQ", dQ, odQ), ("dK", dK, odK), ("dV", dV, odV)):
         hp.assert_close(hp.to_np(g), o, atol, rtol, nm)
     plan.destroy()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name,G,R", [("bert", 116, 42), ("bert", 70, 5), ("bert", 512, 42), ("medium", 300, 42),
+                                      ("skew", 500, 42)])
+@pytest.mark.parametrize("impl_idx", [0, 1], ids=["simt", "tc"])
+def test_global_section_longer_than_the_prefix(name, G, R, impl_idx):
+    # Section 3.1 / Appendix A.2: G = 116, R = 42 with a shorter question: the table tokens at the first
+    # G - |Q| positions of every head's own order are global
+    import torch
+    import paper_2109_04312_b200 as m
+    cfg, rows, cols, info, vals = hp.make_case(name)
+    assert cfg.P < G
+    hv = tables.head_view(cfg)
+    plan = m.mate_plan_bucketed_global(torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda(), cfg.P, G, hv, R)
+    assert np.array_equal(plan.useful_pairs(),
+                          oracle.useful_pairs(rows, cols, cfg.P, hv, radius=R, global_len=G))   # bit exact
+    impl = (m.IMPL_SIMT, m.IMPL_TCGEN05)[impl_idx]
+    scale = 1.0 / np.sqrt(cfg.d)
+    atol, rtol = hp.tol(cfg.dtype)
+    Q, K, V, dO = (hp.to_dev(vals[n], cfg.dtype) for n in ("Q", "K", "V", "dO"))
+    O, LSE = m.mate_attn_fwd(plan, Q, K, V, scale, impl)
+    dQ, dK, dV = m.mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale, impl)
+    torch.cuda.synchronize()
+    plan.status()
+    oO, oLSE = oracle.fwd(vals["Q"], vals["K"], vals["V"], rows, cols, cfg.P, hv, scale, radius=R, global_len=G)
+    want = oracle.bwd(vals["Q"], vals["K"], vals["V"], vals["dO"], rows, cols, cfg.P, hv, scale, radius=R, global_len=G)
+    valid = np.broadcast_to((rows >= 0)[:, None, :], oLSE.shape)
+    hp.assert_close(hp.to_np(O), oO, atol, rtol, "O")
+    hp.assert_close(LSE.cpu().numpy().astype(np.float64)[valid], oLSE[valid], atol, rtol, "LSE")
+    for nm, g, o in zip(("dQ", "dK", "dV"), (dQ, dK, dV), want):
+        hp.assert_close(hp.to_np(g), o, atol, rtol, nm)
+    plan.destroy()
+
+
+@pytest.mark.gpu
+def test_global_section_arguments():
+    import torch
+    import paper_2109_04312_b200 as m
+    cfg, rows, cols, info, _ = hp.make_case("bert")
+    r, c = torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()
+    hv = tables.head_view(cfg)
+    for G, R in ((cfg.P - 1, 42), (cfg.N + 1, 42), (116, 0)):      # below the prefix, beyond N, no radius
+        with pytest.raises(m.MateError) as e:
+            m.mate_plan_bucketed_global(r, c, cfg.P, G, hv, R)
+        assert e.value.status == -1
+    # G = |Q| is the plain bucketed plan
+    p0 = m.mate_plan_bucketed(r, c, cfg.P, hv, 42)
+    p1 = m.mate_plan_bucketed_global(r, c, cfg.P, cfg.P, hv, 42)
+    assert np.array_equal(p0.useful_pairs(), p1.useful_pairs())
+    p0.destroy()
+    p1.destroy()

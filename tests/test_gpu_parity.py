@@ -257,3 +257,26 @@ def test_argument_errors_launch_nothing():
     assert status(lambda: m.mate_attn_bwd(plan, Q, K, V, O, LSE, Q, workspace=tiny_ws)) == -7
     torch.cuda.synchronize()
     plan.destroy()
+
+
+def test_expired_wait_is_reported_once_and_the_plan_stays_usable():
+    # No kernel of the library is made to wait in vain: a one-thread test kernel runs the same bounded
+    # wait with a limit of a few tries on a barrier nothing arrives on, gives up and raises the plan's
+    # time-out word the way the attention kernels would.
+    m = mate()
+    cfg, rows, cols, info, vals = hp.make_case("bert")
+    plan, hv = make_plan(cfg, rows, cols)
+    Q, K, V = (hp.to_dev(vals[n], cfg.dtype) for n in ("Q", "K", "V"))
+    O0, L0 = m.mate_attn_fwd(plan, Q, K, V)
+    torch.cuda.synchronize()
+    plan.status()                                   # nothing has expired so far
+    plan.debug_expire_wait()
+    with pytest.raises(m.MateError) as e:
+        plan.status()
+    assert e.value.status == -5                     # MATE_ERR_TIMEOUT
+    plan.status()                                   # reported once, then clear again
+    O1, L1 = m.mate_attn_fwd(plan, Q, K, V)         # the plan is still good
+    torch.cuda.synchronize()
+    plan.status()
+    assert torch.equal(O0, O1) and torch.equal(L0, L1)
+    plan.destroy()

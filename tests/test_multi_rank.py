@@ -72,3 +72,38 @@ def test_reference_arm_runs_on_rank_zero_only(monkeypatch, capsys):
     monkeypatch.setenv("RANK", "1")
     bench.run_reference(Args(), tables.CONFIGS["tiny"])
     assert capsys.readouterr().out == ""
+
+
+def test_gpus_flag_starts_the_ranks_itself(monkeypatch):
+    """`python bench.py --gpus 4` without a launcher re-executes itself under torch.distributed.run with four
+    ranks on the loopback address; under a launcher (WORLD_SIZE set) it does not."""
+    import bench
+    seen = {}
+
+    def fake_run(cmd):
+        seen["cmd"] = cmd
+        return 0
+
+    assert bench.spawn_ranks(["--gpus", "4", "--steps", "5"], 4, run=fake_run) == 0
+    cmd = seen["cmd"]
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert os.path.basename(cmd[cmd.index("--master-port") + 2]) == "bench.py"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "5"]
+
+    # main(): spawns only when no launcher has set WORLD_SIZE
+    calls = []
+    monkeypatch.setattr(bench, "spawn_ranks", lambda argv, n, run=None: calls.append((argv, n)) or 0)
+    monkeypatch.setattr(bench, "run_mate", lambda args, cfg: calls.append("run_mate"))
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "2"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    try:
+        bench.main()
+    except SystemExit as e:
+        assert e.code == 0
+    assert calls == [(["--gpus", "2"], 2)]
+    calls.clear()
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    bench.main()
+    assert calls == ["run_mate"]
