@@ -258,8 +258,10 @@ def run_mate(args, cfg):
     torch.cuda.synchronize()
     set_bytes = sum(t.numel() * t.element_size() for t in sets[0].values()) + 3 * sets[0]["Q"].numel() * 2
 
+    fwd_impl = mate.IMPL_AUTO | (mate.FLAG_BULK_TILES if args.loader == "bulk" else 0)
+
     def step(d):
-        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, out=d["O"], lse=d["LSE"])
+        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, fwd_impl, out=d["O"], lse=d["LSE"])
         return mate.mate_attn_bwd(plan, d["Q"], d["K"], d["V"], d["O"], d["LSE"], d["dO"], scale)
 
     sampler = ClockSampler(local_rank)
@@ -281,7 +283,7 @@ def run_mate(args, cfg):
     for i in range(K):
         d = sets[i % N_BUFFER_SETS]
         ev[i][0].record()
-        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, out=d["O"], lse=d["LSE"])
+        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, fwd_impl, out=d["O"], lse=d["LSE"])
         ev[i][1].record()
         mate.mate_attn_bwd(plan, d["Q"], d["K"], d["V"], d["O"], d["LSE"], d["dO"], scale)
         ev[i][2].record()
@@ -299,7 +301,7 @@ def run_mate(args, cfg):
     d = sets[0]
     for e in warm_ev:
         e[0].record()
-        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, out=d["O"], lse=d["LSE"])
+        mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, fwd_impl, out=d["O"], lse=d["LSE"])
         e[1].record()
         mate.mate_attn_bwd(plan, d["Q"], d["K"], d["V"], d["O"], d["LSE"], d["dO"], scale)
         e[2].record()
@@ -395,7 +397,7 @@ def run_mate(args, cfg):
                 s_run.wait_event(up_done[j])
                 if i >= 2:
                     s_run.wait_event(down_done[j])    # the results of step i - 2 have left the device
-                mate.mate_attn_fwd(plan, dset["Q"], dset["K"], dset["V"], scale, out=dset["O"], lse=dset["LSE"])
+                mate.mate_attn_fwd(plan, dset["Q"], dset["K"], dset["V"], scale, fwd_impl, out=dset["O"], lse=dset["LSE"])
                 grads[j] = mate.mate_attn_bwd(plan, dset["Q"], dset["K"], dset["V"], dset["O"], dset["LSE"], dset["dO"],
                                               scale)
                 run_done[j].record(s_run)
@@ -446,7 +448,7 @@ def run_mate(args, cfg):
             "config": {"workload": cfg.name, "B": cfg.B, "H": cfg.H, "N": N, "d": cfg.d, "P": cfg.P,
                        "useful_pairs": pairs_all, "dense_pairs": float(world * cfg.B * cfg.H * N * N),
                        "l2": "rotating %d buffer sets of %.0f MB (> 126 MB L2)" % (N_BUFFER_SETS, set_bytes / 1e6),
-                       "plan": "pre-computed, outside the timed region"},
+                       "plan": "pre-computed, outside the timed region", "fwd_loader": args.loader},
             "fwd": {"ms_median": fwd_med, "ms_min": fwd_min, "ms_l2_warm": fwd_warm_ms, "tflops": fwd_tflops,
                     "frac_of_bf16_peak": fwd_tflops / (peaks["bf16_tflops"] * world),
                     "tokens_per_s": tokens_all / (fwd_med * 1e-3)},
@@ -493,6 +495,65 @@ def run_mate(args, cfg):
         dist.destroy_process_group()
 
 
+FWD_TRACE_LABELS = {
+    "softmax warp 0 (half 0)": ["wait S", "wait previous P V", None, "tile: S seen to P handed over", "tiles", "unit set-up",
+                               "epilogue", "total"],
+    "softmax warp 4 (half 1)": ["wait S", "wait previous P V", None, "tile: S seen to P handed over", "tiles", "unit set-up",
+                               "epilogue", "total"],
+    "MMA thread of half 0": ["wait Q", "wait P", "issue Q K^T", "issue P V", "tiles", "wait K/V tile", "wait S free", "total"],
+    "loader warp 10": ["wait for a free buffer", "flush pending copies", "issue copies", "commit and signal", "tiles", None, None,
+                       "total"],
+}
+BWD_TRACE_LABELS = {
+    "arithmetic warp 0": ["wait S/dP", "wait previous gradient MMAs", "arithmetic", "epilogue", "tensor-memory loads", "total",
+                          "signal operands", "tiles"],
+    "arithmetic warp 4": ["wait S/dP", "wait previous gradient MMAs", "arithmetic", "epilogue", "tensor-memory loads", None,
+                          "signal operands", "tiles"],
+    "MMA thread": ["wait row operands", "wait column tile", "wait operands from the warps", "issue gradient MMAs", "issue S/dP",
+                   "wait S/dP read", None, "tiles"],
+    "loader warp": ["wait for a free buffer", None, None, None, None, None, None, None],
+}
+
+
+def run_trace(args, cfg):
+    """Per-role cycle counters of the two tensor-core kernels: builds the profiling variant of the library
+    (-DMATE_TRACE), runs a few steps and prints the mean over the CTAs of every counter, one JSON line."""
+    import ctypes
+    from paper_2109_04312_b200 import build as lib_build
+    os.environ["MATE_LIB"] = lib_build.build(trace=True)
+    import torch
+    import paper_2109_04312_b200 as mate
+    from paper_2109_04312_b200 import api
+    torch.cuda.set_device(0)
+    rows, cols, info = tables.make_structure(cfg, 1234)
+    hv = tables.head_view(cfg)
+    vals = tables.make_values(cfg, info["N"], 5678)
+    plan = mate.mate_plan(torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda(), cfg.P, hv, cfg.n_rows, cfg.n_cols)
+    Q, K, V, dO = (torch.from_numpy(vals[n]).cuda().to(torch.bfloat16) for n in ("Q", "K", "V", "dO"))
+    for _ in range(max(args.warmup, 3)):
+        O, LSE = mate.mate_attn_fwd(plan, Q, K, V)
+        mate.mate_attn_bwd(plan, Q, K, V, O, LSE, dO)
+    torch.cuda.synchronize()
+    plan.status()
+    lib = api._load()
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    out = {"trace": cfg.name, "clock": "SM cycles per CTA, mean over %d CTAs of one launch" % n_sm}
+    for key, fn, labels in (("tc_fwd_kernel", lib.mate_debug_trace, FWD_TRACE_LABELS),
+                            ("tc_bwd_kernel", lib.mate_debug_trace_bwd, BWD_TRACE_LABELS)):
+        buf = np.zeros((256, 4, 8), np.int64)
+        fn.restype = ctypes.c_int
+        assert fn(ctypes.c_void_p(buf.ctypes.data)) == 0
+        buf = buf[:n_sm].astype(np.float64)
+        out[key] = {}
+        for r, (role, names) in enumerate(labels.items()):
+            out[key][role] = {nm: round(float(buf[:, r, i].mean())) for i, nm in enumerate(names) if nm}
+            if "total" in out[key][role]:
+                i = names.index("total")
+                out[key][role]["total of the slowest CTA"] = round(float(buf[:, r, i].max()))
+    print(json.dumps(out), flush=True)
+    plan.destroy()
+
+
 def spawn_ranks(argv, n, run=subprocess.call):
     """`python bench.py --gpus N` without a launcher: start the N ranks here, one per GPU, through
     torch.distributed.run on the loopback address, and return its exit code."""
@@ -513,11 +574,18 @@ def main():
     ap.add_argument("--impl", default="mate", choices=["mate", "reference"])
     ap.add_argument("--workload", default="long", choices=sorted(tables.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--trace", action="store_true",
+                    help="print the per-role cycle counters of the profiling build instead of timing")
+    ap.add_argument("--loader", default="gather", choices=["gather", "bulk"],
+                    help="forward K/V tiles that are contiguous in the tensors: row-by-row gathers like every other "
+                         "tile (default) or bulk tensor copies")
     args = ap.parse_args()
     cfg = tables.CONFIGS[args.workload]
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "mate":
         sys.exit(spawn_ranks(sys.argv[1:], args.gpus))
-    if args.impl == "reference":
+    if args.trace:
+        run_trace(args, cfg)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         args.warmup = max(args.warmup, 3)

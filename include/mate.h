@@ -66,12 +66,14 @@ enum { MATE_IMPL_AUTO = 0, MATE_IMPL_SIMT = 1, MATE_IMPL_TCGEN05 = 2 };
  *                for the head's view), and O and LSE are returned in the same order: what a producer
  *                that writes its projections through the plan's order provides (Section 3.1: the
  *                reordering can be folded into the neighbouring steps).  No gather, no scatter; the
- *                tensor-core kernel then fetches every full tile with bulk tensor copies.  Not for
+ *                tensor-core kernel then fetches every full K/V tile with bulk tensor copies.  Not for
  *                mate_plan_sat plans and not for mate_attn_bwd (MATE_ERR_UNSUPPORTED).
- *   GATHER_ONLY  the tensor-core forward fetches every tile with row-by-row gathers, also those that
- *                are contiguous in the tensors (which otherwise come in by bulk tensor copies): for
- *                comparing the two load paths. */
-enum { MATE_FLAG_VIEW_ORDER = 4, MATE_FLAG_GATHER_ONLY = 8 };
+ *   BULK_TILES   the tensor-core forward fetches the K/V tiles that are contiguous in the tensors -- the
+ *                prefix block of every head and, for a row-major table, every tile of the row view --
+ *                with bulk tensor copies (one per tile and matrix) instead of row-by-row gathers.  Same
+ *                results bit for bit.  Off by default: faster on some workloads, slower on the
+ *                8192-token one. */
+enum { MATE_FLAG_VIEW_ORDER = 4, MATE_FLAG_BULK_TILES = 8 };
 
 const char *mate_status_string(int status);
 
@@ -136,6 +138,20 @@ int mate_plan_bucketed_global(const int32_t *row_ids, const int32_t *col_ids, in
  * B equal entries.  All other arguments, ownership and errors as for mate_plan. */
 int mate_plan_varlen(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix_len,
                      const uint8_t *head_view, int H, int max_row_id, int max_col_id, int radius,
+                     void *stream, mate_plan_t **out);
+
+/* Packed batches: examples of different length stored one behind the other, without padding
+ * (the paper's inputs are a question or a passage followed by a table of any size, Section 3 and
+ * Section 5; the attention of one example never reaches another).  row_ids, col_ids: DEVICE int32
+ * [T], example b owning the tokens cu_seqlens[b] .. cu_seqlens[b + 1] - 1; cu_seqlens: HOST int32
+ * [B + 1], cu_seqlens[0] = 0, non-decreasing, cu_seqlens[B] = T; prefix_len: HOST int32 [B],
+ * 0 <= prefix_len[b] <= length of example b.  Negative ids inside an example still mark padding.
+ * With such a plan every tensor of mate_attn_fwd / mate_attn_bwd / mate_attn_bwd_noalloc is
+ * [H, T, d] (LSE [H, T]) in place of [B, H, N, d] ([B, H, N]); the plan's N (mate_plan_get,
+ * mate_attn_workspace_bytes) is the longest example.  The exact pattern only; MATE_FLAG_VIEW_ORDER
+ * and mate_cell_mean return MATE_ERR_UNSUPPORTED.  Ownership and errors as for mate_plan. */
+int mate_plan_packed(const int32_t *row_ids, const int32_t *col_ids, int B, const int32_t *cu_seqlens,
+                     const int32_t *prefix_len, const uint8_t *head_view, int H, int max_row_id, int max_col_id,
                      void *stream, mate_plan_t **out);
 
 /* Plan of the head-independent pattern that the paper describes for its closest comparison system

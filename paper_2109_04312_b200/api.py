@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libmate.so")
 
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
-FLAG_VIEW_ORDER, FLAG_GATHER_ONLY = 4, 8   # or-ed to the implementation choice (see mate.h)
+FLAG_VIEW_ORDER, FLAG_BULK_TILES = 4, 8   # or-ed to the implementation choice (see mate.h)
 VIEW_ROW, VIEW_COL = 0, 1
 _BF16, _F32 = 0, 1
 
@@ -23,7 +23,9 @@ class MateError(RuntimeError):
 
 
 def library_path() -> str:
-    return _LIB_PATH
+    """MATE_LIB (read when the library is first loaded) selects another build of the same library:
+    the profiling build, libmate_trace.so."""
+    return os.environ.get("MATE_LIB") or _LIB_PATH
 
 
 def _load():
@@ -31,11 +33,12 @@ def _load():
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(_LIB_PATH):
+    path = library_path()
+    if not os.path.exists(path):
         raise ImportError(
             "libmate.so is not built: run `python -m paper_2109_04312_b200.build` "
             "(needs nvcc); there is no CPU or PyTorch fallback")
-    lib = C.CDLL(_LIB_PATH)
+    lib = C.CDLL(path)
     vp, i32, u32, f32, sz = C.c_void_p, C.c_int, C.c_uint, C.c_float, C.c_size_t
     lib.mate_status_string.restype = C.c_char_p
     lib.mate_status_string.argtypes = [i32]
@@ -45,6 +48,8 @@ def _load():
     lib.mate_plan_bucketed.argtypes = [vp, vp, i32, i32, i32, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_varlen.restype = i32
     lib.mate_plan_varlen.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
+    lib.mate_plan_packed.restype = i32
+    lib.mate_plan_packed.argtypes = [vp, vp, i32, vp, vp, vp, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_bucketed_global.restype = i32
     lib.mate_plan_bucketed_global.argtypes = [vp, vp, i32, i32, vp, vp, vp, i32, i32, i32, i32, vp, C.POINTER(vp)]
     lib.mate_plan_sat.restype = i32
@@ -111,7 +116,18 @@ class Plan:
         self.B, self.N, self.P, self.H = B, N, P, H
         self.max_id = (max_row_id, max_col_id)
         self.device = device
+        self.T = None          # packed plans: total number of tokens (tensors are [H, T, d])
         self._ws = {}
+
+    def _split(self, Q):
+        """Checks a tensor's shape against the plan; returns (d, shape of the row statistic)."""
+        if self.T is not None:
+            if Q.dim() != 3 or tuple(Q.shape[:2]) != (self.H, self.T):
+                raise ValueError("a packed plan takes [H, T, d] tensors")
+            return Q.shape[2], (self.H, self.T)
+        if Q.dim() != 4 or tuple(Q.shape[:3]) != (self.B, self.H, self.N):
+            raise ValueError("tensor shapes do not match the plan")
+        return Q.shape[3], (self.B, self.H, self.N)
 
     def get(self, view):
         """(perm, inv_perm, seg_off) of one view as numpy int32 arrays."""
@@ -149,6 +165,34 @@ class Plan:
 def mate_plan_bucketed(row_ids, col_ids, prefix_len, head_view, radius, max_row_id=None, max_col_id=None) -> Plan:
     """Plan of the bucketed variant (see mate_plan_bucketed in mate.h); radius = 0 is the exact pattern."""
     return mate_plan(row_ids, col_ids, prefix_len, head_view, max_row_id, max_col_id, radius=radius)
+
+
+def mate_plan_packed(row_ids, col_ids, cu_seqlens, prefix_lens, head_view, max_row_id=None, max_col_id=None) -> Plan:
+    """Plan of a packed batch (see mate_plan_packed in mate.h): row_ids, col_ids are int32 CUDA tensors [T],
+    example b owning the tokens cu_seqlens[b] .. cu_seqlens[b + 1] - 1; Q, K, V, O and the gradients are then
+    [H, T, d] and LSE is [H, T]."""
+    if row_ids.dtype != torch.int32 or col_ids.dtype != torch.int32 or row_ids.shape != col_ids.shape \
+            or row_ids.dim() != 1:
+        raise ValueError("row_ids / col_ids must be int32 tensors of the same [T] shape")
+    cu = np.ascontiguousarray(np.asarray(cu_seqlens, dtype=np.int32))
+    pf = np.ascontiguousarray(np.asarray(prefix_lens, dtype=np.int32))
+    B = int(pf.shape[0])
+    if cu.shape != (B + 1,) or int(cu[-1]) != int(row_ids.shape[0]):
+        raise ValueError("cu_seqlens must have B + 1 entries and end at T")
+    hv = np.ascontiguousarray(np.asarray(head_view, dtype=np.uint8))
+    if max_row_id is None:
+        max_row_id = max(int(row_ids.max().item()), 0) if row_ids.numel() else 0
+    if max_col_id is None:
+        max_col_id = max(int(col_ids.max().item()), 0) if col_ids.numel() else 0
+    handle = C.c_void_p()
+    with torch.cuda.device(row_ids.device):
+        _check(_load().mate_plan_packed(_dev(row_ids, "row_ids"), _dev(col_ids, "col_ids"), B, cu.ctypes.data,
+                                        pf.ctypes.data, hv.ctypes.data, int(hv.shape[0]), int(max_row_id),
+                                        int(max_col_id), _stream(), C.byref(handle)), "mate_plan_packed")
+    n_max = max(int(np.diff(cu).max()), 1)
+    plan = Plan(handle, B, n_max, pf.tolist(), int(hv.shape[0]), int(max_row_id), int(max_col_id), row_ids.device)
+    plan.T = int(cu[-1])
+    return plan
 
 
 def mate_plan_varlen(row_ids, col_ids, prefix_lens, head_view, radius=0, max_row_id=None, max_col_id=None) -> Plan:
@@ -246,15 +290,16 @@ def _workspace(plan, nbytes, key):
 
 
 def mate_attn_fwd(plan, Q, K, V, scale=None, impl=IMPL_AUTO, out=None, lse=None, workspace=None):
-    """Q, K, V: [B, H, N, d] CUDA tensors (bf16 or f32).  Returns (O, LSE) in original token order."""
-    B, H, N, d = Q.shape
-    if (B, H, N) != (plan.B, plan.H, plan.N) or K.shape != Q.shape or V.shape != Q.shape:
+    """Q, K, V: [B, H, N, d] CUDA tensors (bf16 or f32), or [H, T, d] for a packed plan.  Returns (O, LSE)
+    in original token order."""
+    d, stat_shape = plan._split(Q)
+    if K.shape != Q.shape or V.shape != Q.shape:
         raise ValueError("tensor shapes do not match the plan")
     dt = _dtype_code(Q)
     if scale is None:
         scale = 1.0 / float(d) ** 0.5
     O = torch.empty_like(Q) if out is None else out
-    LSE = torch.empty((B, H, N), dtype=torch.float32, device=Q.device) if lse is None else lse
+    LSE = torch.empty(stat_shape, dtype=torch.float32, device=Q.device) if lse is None else lse
     need, _ = mate_attn_workspace_bytes(plan, d, dt, impl)
     ws = workspace if workspace is not None else _workspace(plan, need, "fwd")
     with torch.cuda.device(Q.device):
@@ -268,9 +313,7 @@ def mate_attn_fwd(plan, Q, K, V, scale=None, impl=IMPL_AUTO, out=None, lse=None,
 
 def mate_attn_bwd(plan, Q, K, V, O, LSE, dO, scale=None, impl=IMPL_AUTO, workspace=None):
     """Returns (dQ, dK, dV)."""
-    B, H, N, d = Q.shape
-    if (B, H, N) != (plan.B, plan.H, plan.N):
-        raise ValueError("tensor shapes do not match the plan")
+    d, _ = plan._split(Q)
     for t in (K, V, O, dO):
         if t.shape != Q.shape or t.dtype != Q.dtype:
             raise ValueError("K, V, O, dO must match Q in shape and dtype")
@@ -316,9 +359,7 @@ def mate_attn_bwd_noalloc(plan, Q, K, V, O, LSE, dO, dQ, dK, dV, scale=None):
     framework owns every byte of the device): the caller passes the three output tensors and the
     library uses its built-in scratch array, so neither this function nor the C entry point
     allocates anything.  B*H*N is limited to 1,048,576.  Calls must not overlap on the GPU."""
-    B, H, N, d = Q.shape
-    if (B, H, N) != (plan.B, plan.H, plan.N):
-        raise ValueError("tensor shapes do not match the plan")
+    d, _ = plan._split(Q)
     for t in (K, V, O, dO, dQ, dK, dV):
         if t.shape != Q.shape or t.dtype != Q.dtype:
             raise ValueError("K, V, O, dO, dQ, dK, dV must match Q in shape and dtype")

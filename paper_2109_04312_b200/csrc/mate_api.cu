@@ -269,6 +269,7 @@ int mate_plan_destroy(mate_plan_t *plan) {
     if (!plan) return MATE_OK;
     for (int s = 0; s < 2; ++s) mate_plan_destroy(plan->sub[s]);
     if (plan->pair_ids_dev) cudaFree(plan->pair_ids_dev);
+    if (plan->tok_off_dev) cudaFree(plan->tok_off_dev);
     if (plan->dev_block) cudaFree(plan->dev_block);
     if (plan->work_block) cudaFree(plan->work_block);
     delete plan;
@@ -312,6 +313,52 @@ int mate_plan_bucketed_global(const int32_t *row_ids, const int32_t *col_ids, in
         if (global_len[b] < prefix_len[b] || global_len[b] > N) return MATE_ERR_INVALID_ARG;
     return build_plan(row_ids, col_ids, B, N, prefix_len, global_len, head_view, H, max_row_id, max_col_id, radius,
                       mate::kBoundsOwn, 1, stream, out);
+}
+
+/* Packed batches: the examples lie one behind the other on a common token axis.  The plan itself is the
+ * padded one over N = the longest example (small integer arrays); what changes is where the kernels
+ * find an example's rows in the tensors, and that positions behind an example's end do not exist. */
+int mate_plan_packed(const int32_t *row_ids, const int32_t *col_ids, int B, const int32_t *cu_seqlens,
+                     const int32_t *prefix_len, const uint8_t *head_view, int H, int max_row_id, int max_col_id,
+                     void *stream, mate_plan_t **out) {
+    if (out) *out = nullptr;
+    if (!row_ids || !col_ids || !cu_seqlens || !prefix_len || !head_view || !out || B <= 0 || H <= 0)
+        return MATE_ERR_INVALID_ARG;
+    if (cu_seqlens[0] != 0) return MATE_ERR_INVALID_ARG;
+    int n_max = 1;
+    std::vector<int32_t> off_len((size_t)2 * B);
+    for (int b = 0; b < B; ++b) {
+        const int len = cu_seqlens[b + 1] - cu_seqlens[b];
+        if (len < 0 || prefix_len[b] < 0 || prefix_len[b] > len) return MATE_ERR_INVALID_ARG;
+        n_max = std::max(n_max, len);
+        off_len[b] = cu_seqlens[b];
+        off_len[B + b] = len;
+    }
+    const int T = cu_seqlens[B];
+    cudaStream_t st = (cudaStream_t)stream;
+    int32_t *off_dev = nullptr, *ids = nullptr;
+    const size_t BN = (size_t)B * n_max;
+    if (cudaMalloc(&off_dev, sizeof(int32_t) * 2 * B) != cudaSuccess || cudaMalloc(&ids, sizeof(int32_t) * 2 * BN) != cudaSuccess) {
+        cudaGetLastError();
+        if (off_dev) cudaFree(off_dev);
+        return MATE_ERR_NOMEM;
+    }
+    bool ok = cudaMemcpyAsync(off_dev, off_len.data(), sizeof(int32_t) * 2 * B, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && mate::launch_unpack_ids(row_ids, col_ids, B, n_max, off_dev, off_dev + B, ids, ids + BN, st) == cudaSuccess;
+    mate_plan_t *pl = nullptr;
+    int rc = ok ? build_plan(ids, ids + BN, B, n_max, prefix_len, nullptr, head_view, H, max_row_id, max_col_id, 0,
+                             mate::kBoundsOwn, 1, stream, &pl)
+                : MATE_ERR_CUDA;
+    cudaFree(ids);  // build_plan has waited for its kernels
+    if (rc != MATE_OK) {
+        cudaFree(off_dev);
+        return rc;
+    }
+    pl->T = T;
+    pl->tok_off_dev = off_dev;
+    pl->len_dev = off_dev + B;
+    *out = pl;
+    return MATE_OK;
 }
 
 /* The head-independent pattern: three passes over plans the ordinary kernels can run (see mate.h).
@@ -543,7 +590,7 @@ static int check_common(const mate_plan_t *plan, int d, int dtype, unsigned flag
     if (dtype != MATE_BF16 && dtype != MATE_F32) return MATE_ERR_UNSUPPORTED;
     if (d <= 0 || d % 8 != 0 || d > 128) return MATE_ERR_UNSUPPORTED;
     const unsigned impl = flags & 3u;
-    if (impl == 3u || (flags & ~(3u | MATE_FLAG_VIEW_ORDER | MATE_FLAG_GATHER_ONLY))) return MATE_ERR_INVALID_ARG;
+    if (impl == 3u || (flags & ~(3u | MATE_FLAG_VIEW_ORDER | MATE_FLAG_BULK_TILES))) return MATE_ERR_INVALID_ARG;
     const bool tc_ok = mate::tc_supported(d, dtype);
     if (impl == MATE_IMPL_TCGEN05 && !tc_ok) return MATE_ERR_UNSUPPORTED;
     *use_tc = (impl == MATE_IMPL_TCGEN05) || (impl == MATE_IMPL_AUTO && tc_ok);
@@ -569,7 +616,7 @@ int mate_attn_workspace_bytes(const mate_plan_t *plan, int d, int dtype, unsigne
     bool use_tc = false;
     int rc = check_common(plan, d, dtype, flags, &use_tc);
     if (rc != MATE_OK) return rc;
-    const size_t rows = (size_t)plan->B * plan->H * plan->N;
+    const size_t rows = plan->n_rows();
     size_t f = pass_fwd_bytes(plan, d, use_tc), b = pass_bwd_bytes(plan, use_tc);
     if (plan->sub[0]) {
         f += 2 * (align_up(rows * d * elem_bytes(dtype), 256) + align_up(rows * sizeof(float), 256));
@@ -606,11 +653,11 @@ int mate_attn_fwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     mate_attn_workspace_bytes(plan, d, dtype, use_tc ? MATE_IMPL_TCGEN05 : MATE_IMPL_SIMT, &need, nullptr);
     if (need > 0 && (!workspace || workspace_bytes < need)) return MATE_ERR_WORKSPACE;
     if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MATE_ERR_ALIGNMENT;
-    if ((flags & MATE_FLAG_VIEW_ORDER) && plan->sub[0]) return MATE_ERR_UNSUPPORTED;  // the passes use different orders
+    if ((flags & MATE_FLAG_VIEW_ORDER) && (plan->sub[0] || plan->T)) return MATE_ERR_UNSUPPORTED;
     rc = fwd_pass(plan, use_tc, Q, K, V, d, dtype, scale, O, LSE, workspace, flags, st);
     if (rc != MATE_OK || !plan->sub[0]) return rc;
     // row-or-column pattern: the two passes over the rest of the column, then the merge
-    const size_t rows = (size_t)plan->B * plan->H * plan->N;
+    const size_t rows = plan->n_rows();
     const size_t o_bytes = align_up(rows * d * elem_bytes(dtype), 256), l_bytes = align_up(rows * sizeof(float), 256);
     char *w = (char *)workspace + pass_fwd_bytes(plan, d, use_tc);
     void *Os[2];
@@ -657,7 +704,7 @@ int mate_attn_bwd(const mate_plan_t *plan, const void *Q, const void *K, const v
     // pairs.  The two column passes are each other's transpose (keys in front of / behind the own
     // cell), and the kernels take a plan's key ranges for the query side and for the key side alike;
     // run on both plans and summed, every pair is still counted once on each side.
-    const size_t n = (size_t)plan->B * plan->H * plan->N * d;
+    const size_t n = plan->n_rows() * d;
     const size_t g_bytes = align_up(n * elem_bytes(dtype), 256);
     char *w = (char *)workspace + pass_bwd_bytes(plan, use_tc);
     void *g[2][3];

@@ -88,6 +88,7 @@ struct Params {
     const uint8_t *head_view;
     const FwdUnit *units;
     int n_units, N, H;
+    TensorRows tr;         // where (example, head) starts in the tensors
     float scale, scale_log2;
     int32_t *status;
     int32_t *counter;      // next work item (zeroed before the launch)
@@ -311,13 +312,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
             const FwdUnit &un = x.un;
             const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
             const int32_t *perm = vp.perm + (size_t)un.b * p.N;
-            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const size_t bh = p.tr.base(un.b, un.h);
             const bool row_valid = r < x.rows_h;
             const int t_row = x.row0 + min(r, x.rows_h - 1);  // rows past the end shadow the last one
             const int orig = perm[t_row];
 
             if (x.n_tiles == 0) {  // padding rows: zero gradients
-                if (row_valid && cq == 0) {
+                if (row_valid && cq == 0 && p.tr.exists(un.b, orig)) {
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
                         if (!x.key_side) reinterpret_cast<uint4 *>(p.dQ + (bh + orig) * 64)[q] = make_uint4(0, 0, 0, 0);
@@ -745,7 +746,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_bwd_kernel(const Params p) {
             const FwdUnit &un = x.un;
             const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
             const int32_t *perm = vp.perm + (size_t)un.b * p.N;
-            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const size_t bh = p.tr.base(un.b, un.h);
             const __nv_bfloat16 *Ra_bh = (x.key_side ? p.K : p.Q) + bh * 64, *Rb_bh = (x.key_side ? p.V : p.dO) + bh * 64;
             const __nv_bfloat16 *Ca_bh = (x.key_side ? p.Q : p.K) + bh * 64, *Cb_bh = (x.key_side ? p.dO : p.V) + bh * 64;
 
@@ -828,7 +829,7 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
            cudaStream_t stream) {
     if (plan->n_bwd_units == 0) return MATE_OK;
     if (g_smem_attr.ensure((const void *)tc_bwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
-    const size_t bhn = (size_t)plan->B * plan->H * plan->N;
+    const size_t bhn = plan->n_rows();
     uint8_t *ws = (uint8_t *)workspace;
     Params p;
     p.Q = (const __nv_bfloat16 *)Q;
@@ -849,6 +850,7 @@ int tc_bwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.n_units = plan->n_bwd_units;
     p.N = plan->N;
     p.H = plan->H;
+    p.tr = plan->rows();
     p.scale = scale;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = plan->status_dev;

@@ -74,6 +74,7 @@ extern "C" int mate_cell_mean(const mate_plan_t *plan, const float *logits, cons
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return MATE_ERR_CUDA;
     if (dev != plan->device) return MATE_ERR_INVALID_ARG;
+    if (plan->T) return MATE_ERR_UNSUPPORTED;  // packed batches: not here
     const int n_rows = plan->view[0].max_id + 1, n_cols = plan->view[1].max_id + 1;
     dim3 grid((n_rows + mate::kWarpsPerBlock - 1) / mate::kWarpsPerBlock, plan->B);
     mate::cell_mean_kernel<<<grid, 32 * mate::kWarpsPerBlock, 0, (cudaStream_t)stream>>>(

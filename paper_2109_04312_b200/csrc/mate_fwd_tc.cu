@@ -82,8 +82,8 @@ constexpr int kSchedReaders = kSoftmaxWarps + kMmaWarps + kLoadWarps;
 static_assert(kStages <= 5, "barrier slots");
 
 struct Params {
-    // 2-D tensor maps over Q, K, V seen as [B H N rows, 64 columns]: boxes of 128 rows, 128-byte swizzle
-    CUtensorMap tmQ, tmK, tmV;
+    // 2-D tensor maps over K and V seen as [B H N rows, 64 columns]: boxes of 128 rows, 128-byte swizzle
+    CUtensorMap tmK, tmV;
     int use_tma;     // 0: every tile is gathered row by row
     int view_order;  // 1: Q, K, V, O and LSE are laid out in each head's own order (no gather, no scatter)
     const __nv_bfloat16 *Q, *K, *V;
@@ -94,6 +94,7 @@ struct Params {
     const FwdUnit *units;
     int n_units;
     int N, H;
+    TensorRows tr;     // where (example, head) starts in the tensors
     float scale_log2;  // scale * log2(e)
     int32_t *status;
     int32_t *counters;
@@ -313,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_consta
             if (rows_h == 0) continue;
             const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
             const int32_t *perm = vp.perm + (size_t)un.b * p.N;
-            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const size_t bh = p.tr.base(un.b, un.h);
             const bool row_valid = r < rows_h;
             const int t_row = un.q0 + h * kTile + min(r, rows_h - 1);  // rows past the end shadow the last one
             const int orig = p.view_order ? t_row : perm[t_row];
@@ -321,7 +322,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_consta
             const int h_lo = h ? un.lo[1] : un.lo[0], h_hi = h ? un.hi[1] : un.hi[0];  // segments of this half's rows
 
             if (n_tiles == 0) {  // padding rows: O = 0, LSE = -inf
-                if (row_valid) {
+                if (row_valid && p.tr.exists(un.b, orig)) {
                     uint4 *dst = reinterpret_cast<uint4 *>(p.O + (bh + orig) * 64);
 #pragma unroll
                     for (int c = 0; c < 8; ++c) dst[c] = make_uint4(0, 0, 0, 0);
@@ -843,9 +844,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_consta
             if (n_tiles == 0) continue;
             const ViewPlan &vp = p.head_view[un.h] ? p.colv : p.rowv;
             const int32_t *perm = p.view_order ? nullptr : vp.perm + (size_t)un.b * p.N;
-            const size_t bh = ((size_t)un.b * p.H + un.h) * p.N;
+            const size_t bh = p.tr.base(un.b, un.h);
             const __nv_bfloat16 *Qbh = p.Q + bh * 64, *Kbh = p.K + bh * 64, *Vbh = p.V + bh * 64;
-            // Rows of the order that sit in place in the tensors ([0, ident)): a full tile inside that
+            // Rows of the order that sit in place in the tensors ([0, ident)): a full K/V tile inside that
             // range is one contiguous [128, 64] box and comes in by one bulk tensor copy per matrix
             // (issued by one thread, completing on the tile's barrier by byte count) instead of 2 x 1024
             // gathered 16-byte copies.  That is the prefix block of every unit and, for a row-major
@@ -854,33 +855,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_consta
 
             const int qb = unit_cnt & 1;
             if (!(alive = wait_free(bars + 8 * (kBarQEmpty + qb), ((unit_cnt >> 1) & 1) ^ 1))) break;
-            {
-                const uint32_t bar_q = bars + 8 * (kBarQFull + qb);
-                bool gathered = false;
-                for (int h = 0; h < 2; ++h) {
-                    const int rows_h = rows_of_half(un, h);
-                    if (rows_h == 0) continue;
-                    const int r0 = un.q0 + h * kTile;
-                    const uint32_t dst = base + kOffQ + (qb * 2 + h) * kTileBytes;
-                    if (rows_h == kTile && r0 + kTile <= ident) {
-                        if (ltid == 0) {
-                            mbar_expect_tx(bar_q, kTileBytes);
-                            tma_load_2d(dst, &p.tmQ, 0, (int)bh + r0, bar_q);
-                        }
-                    } else {
-                        int idx[kPasses];
-                        load_indices(idx, perm, r0, kTile, rows_h - 1, ltid);
-                        copy_rows(dst, Qbh, idx, ltid);
-                        gathered = true;
-                    }
-                }
-                if (gathered) {
-                    commit_and_signal(bar_q);
-                } else {
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_q);
+            // (Q tiles are always gathered: fetching them with bulk copies as well measured slower.)
+            for (int h = 0; h < 2; ++h) {
+                const int rows_h = rows_of_half(un, h);
+                if (rows_h > 0) {
+                    int idx[kPasses];
+                    load_indices(idx, perm, un.q0 + h * kTile, kTile, rows_h - 1, ltid);
+                    copy_rows(base + kOffQ + (qb * 2 + h) * kTileBytes, Qbh, idx, ltid);
                 }
             }
+            commit_and_signal(bars + 8 * (kBarQFull + qb));
             ++unit_cnt;
 
             for (int i = 0; i < n_tiles; ++i) {
@@ -985,10 +969,11 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     if (plan->n_fwd_units == 0) return MATE_OK;
     if (g_smem_attr.ensure((const void *)tc_fwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
     Params p;
-    const size_t rows = (size_t)plan->B * plan->H * plan->N;
-    // bulk tensor copies for the tiles that are contiguous in the caller's tensors; without the driver
-    // entry point (or with MATE_FLAG_GATHER_ONLY) every tile is gathered row by row
-    p.use_tma = !(flags & MATE_FLAG_GATHER_ONLY) && rows < (size_t(1) << 31) && make_row_map(&p.tmQ, Q, rows) &&
+    const size_t rows = plan->n_rows();
+    // On request (and always for tensors in view order): bulk tensor copies for the K/V tiles that are
+    // contiguous in the caller's tensors.  By default every tile is gathered row by row, which measured
+    // faster on the 8192-token workload; without the driver entry point there is no choice.
+    p.use_tma = (flags & (MATE_FLAG_BULK_TILES | MATE_FLAG_VIEW_ORDER)) && rows < (size_t(1) << 31) &&
                 make_row_map(&p.tmK, K, rows) && make_row_map(&p.tmV, V, rows);
     p.view_order = (flags & MATE_FLAG_VIEW_ORDER) ? 1 : 0;
     p.Q = (const __nv_bfloat16 *)Q;
@@ -1003,6 +988,7 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     p.n_units = plan->n_fwd_units;
     p.N = plan->N;
     p.H = plan->H;
+    p.tr = plan->rows();
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = plan->status_dev;
     p.counters = plan->fwd_counters_dev;

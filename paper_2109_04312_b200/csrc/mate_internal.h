@@ -42,6 +42,23 @@ static_assert(sizeof(FwdUnit) == 64, "FwdUnit is read as four 16-byte words");
 // bytes of one partial result: 256 rows x (64 fp32 + running max + row sum)
 constexpr size_t kPartialBytes = (size_t)kUnitRows * (64 + 2) * sizeof(float);
 
+// Where the rows of example b, head h start in the caller's tensors (in rows of d elements), and how
+// far an example reaches.  Padded layout [B, H, N, d]: (b H + h) N, every example N positions long.
+// Packed layout [H, T, d] (mate_plan_packed: the examples one behind the other, no padding between
+// them): h T + tok_off[b], example b being len[b] positions long; positions at and beyond len[b] of
+// the plan's padded view of the example do not exist in the tensors and are never written.
+struct TensorRows {
+    const int32_t *tok_off = nullptr;  // device [B]; null = padded layout
+    const int32_t *len = nullptr;      // device [B]; null = padded layout
+    int H = 0, N = 0, T = 0;
+#ifdef __CUDACC__
+    __device__ __forceinline__ size_t base(int b, int h) const {
+        return tok_off ? (size_t)h * T + tok_off[b] : ((size_t)b * H + h) * N;
+    }
+    __device__ __forceinline__ bool exists(int b, int pos) const { return !len || pos < len[b]; }
+#endif
+};
+
 struct ViewPlan {
     int32_t *perm = nullptr;      // [B, N]   view position -> original position
     int32_t *inv_perm = nullptr;  // [B, N]
@@ -73,6 +90,19 @@ struct mate_plan_s {
     // over the rest of the token's column in front of / behind its own cell
     mate_plan_s *sub[2] = {nullptr, nullptr};
     int32_t *pair_ids_dev = nullptr;     // ids of the sub-plans (owned by the main plan)
+    // packed layout (mate_plan_packed): start and length of every example on the common token axis
+    int T = 0;                           // total tokens; 0 = padded layout
+    int32_t *tok_off_dev = nullptr, *len_dev = nullptr;  // [B] each (one allocation, owned by the plan)
+    mate::TensorRows rows() const {
+        mate::TensorRows r;
+        r.tok_off = tok_off_dev;
+        r.len = len_dev;
+        r.H = H;
+        r.N = N;
+        r.T = T;
+        return r;
+    }
+    size_t n_rows() const { return T ? (size_t)H * T : (size_t)B * H * N; }  // rows of a [.., d] tensor
     std::vector<uint8_t> head_view;      // host copy
     uint8_t *head_view_dev = nullptr;    // [H]
     mate::ViewPlan view[2];
@@ -126,6 +156,8 @@ cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, 
                                 int radius, int bounds_mode, int group,
                                 const ViewPlan &rowv, const ViewPlan &colv, int32_t *n_valid, int32_t *status,
                                 cudaStream_t stream);
+cudaError_t launch_unpack_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *tok_off,
+                              const int32_t *len, int32_t *rows_out, int32_t *cols_out, cudaStream_t stream);
 cudaError_t launch_pair_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix,
                             int n_row_ids, int32_t *out, cudaStream_t stream);
 

@@ -186,6 +186,18 @@ cudaError_t launch_plan_kernels(const int32_t *row_ids, const int32_t *col_ids, 
 }
 
 namespace {
+// packed ids (examples one behind the other) -> one padded row of N ids per example, -1 behind its end
+__global__ void unpack_ids_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, size_t n, int N,
+                                  const int32_t *__restrict__ tok_off, const int32_t *__restrict__ len,
+                                  int32_t *__restrict__ rows_out, int32_t *__restrict__ cols_out) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int b = (int)(i / N), k = (int)(i % N);
+    const bool in = k < len[b];
+    rows_out[i] = in ? row_ids[tok_off[b] + k] : -1;
+    cols_out[i] = in ? col_ids[tok_off[b] + k] : -1;
+}
+
 // ids of the two extra passes of the row-or-column pattern: (column, row) pairs as one id,
 // column-major, for table tokens; -1 (treated as padding by those passes) for everything else
 __global__ void pair_ids_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col_ids, size_t n,
@@ -197,6 +209,14 @@ __global__ void pair_ids_kernel(const int32_t *__restrict__ row_ids, const int32
     out[i] = (k >= prefix[b] && r >= 0 && c >= 0) ? c * n_row_ids + r : -1;
 }
 }  // namespace
+
+cudaError_t launch_unpack_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *tok_off,
+                              const int32_t *len, int32_t *rows_out, int32_t *cols_out, cudaStream_t stream) {
+    const size_t n = (size_t)B * N;
+    unpack_ids_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(row_ids, col_ids, n, N, tok_off, len, rows_out,
+                                                                       cols_out);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_pair_ids(const int32_t *row_ids, const int32_t *col_ids, int B, int N, const int32_t *prefix,
                             int n_row_ids, int32_t *out, cudaStream_t stream) {

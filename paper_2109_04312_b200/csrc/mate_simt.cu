@@ -75,17 +75,18 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 simt_fwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__restrict__ V,
                 T *__restrict__ O, float *__restrict__ LSE, ViewPlan rowv, ViewPlan colv,
                 const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
-                const int32_t *__restrict__ prefix, int d, float scale, int view_order) {
+                const int32_t *__restrict__ prefix, int d, float scale, int view_order, TensorRows tr) {
     __shared__ float s_q[kWarpsPerBlock][kMaxD];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kWarpsPerBlock + warp;
-    const int h = blockIdx.y, b = blockIdx.z, H = gridDim.y;
+    const int h = blockIdx.y, b = blockIdx.z;
     if (t >= N) return;
     const RowCtx c = row_ctx(rowv, colv, head_view, n_valid, b, h, N);
-    const size_t bh = ((size_t)b * H + h) * N;
+    const size_t bh = tr.base(b, h);
     const int k = view_order ? t : c.perm[t];  // view order: the tensors are laid out in the head's own order
     T *o_row = O + (bh + k) * d;
     if (t >= c.n_valid) {  // padding query row
+        if (!tr.exists(b, k)) return;  // packed layout: beyond the example's end there is no such row
         for (int e = lane; e < d; e += 32) from_f(o_row[e], 0.f);
         if (lane == 0) LSE[bh + k] = -INFINITY;
         return;
@@ -162,19 +163,20 @@ simt_bwd_kernel(const T *__restrict__ Q, const T *__restrict__ K, const T *__res
                 const float *__restrict__ D, T *__restrict__ dQ, T *__restrict__ dK,
                 T *__restrict__ dV, ViewPlan rowv, ViewPlan colv,
                 const uint8_t *__restrict__ head_view, const int32_t *__restrict__ n_valid, int N,
-                const int32_t *__restrict__ prefix, int d, float scale) {
+                const int32_t *__restrict__ prefix, int d, float scale, TensorRows tr) {
     __shared__ float s_a[kWarpsPerBlock][kMaxD];  // own q (dQ) or own k (dK/dV)
     __shared__ float s_b[kWarpsPerBlock][kMaxD];  // own dO (dQ) or own v (dK/dV)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kWarpsPerBlock + warp;
-    const int h = blockIdx.y, b = blockIdx.z, H = gridDim.y;
+    const int h = blockIdx.y, b = blockIdx.z;
     if (t >= N) return;
     const RowCtx c = row_ctx(rowv, colv, head_view, n_valid, b, h, N);
-    const size_t bh = ((size_t)b * H + h) * N;
+    const size_t bh = tr.base(b, h);
     const int own = c.perm[t];
     T *out0 = (kDKV ? dK : dQ) + (bh + own) * d;
     T *out1 = kDKV ? dV + (bh + own) * d : nullptr;
     if (t >= c.n_valid) {
+        if (!tr.exists(b, own)) return;  // packed layout: beyond the example's end there is no such row
         for (int e = lane; e < d; e += 32) {
             from_f(out0[e], 0.f);
             if (kDKV) from_f(out1[e], 0.f);
@@ -252,7 +254,7 @@ int simt_fwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *
     dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
     simt_fwd_kernel<T><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (T *)O, LSE, pl->view[0], pl->view[1],
-        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale, view_order);
+        pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale, view_order, pl->rows());
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
@@ -261,16 +263,16 @@ int simt_bwd_t(const mate_plan_t *pl, const void *Q, const void *K, const void *
                const float *LSE, const void *dO, int d, float scale, void *dQ, void *dK, void *dV,
                void *ws, cudaStream_t st) {
     float *D = (float *)ws;
-    const size_t rows = (size_t)pl->B * pl->H * pl->N;
+    const size_t rows = pl->n_rows();
     simt_rowdot_kernel<T><<<(unsigned)((rows + kWarpsPerBlock - 1) / kWarpsPerBlock),
                             kWarpsPerBlock * 32, 0, st>>>((const T *)dO, (const T *)O, D, rows, d);
     dim3 grid((pl->N + kWarpsPerBlock - 1) / kWarpsPerBlock, pl->H, pl->B);
     simt_bwd_kernel<T, false><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
-        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale);
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale, pl->rows());
     simt_bwd_kernel<T, true><<<grid, kWarpsPerBlock * 32, 0, st>>>(
         (const T *)Q, (const T *)K, (const T *)V, (const T *)dO, LSE, D, (T *)dQ, (T *)dK, (T *)dV,
-        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale);
+        pl->view[0], pl->view[1], pl->head_view_dev, pl->n_valid_dev, pl->N, pl->global_dev, d, scale, pl->rows());
     return cudaGetLastError() == cudaSuccess ? MATE_OK : MATE_ERR_CUDA;
 }
 
