@@ -1,6 +1,6 @@
-// Per-view token order (Section 3.1: every head traverses the table in its own row-order or
-// column-order, "data-dependent but deterministic"): a stable counting sort of the positions by
-// (prefix, table id, padding).  One CTA per (example, view); integer work only.
+// Per-view token order (Section 3.1: every head traverses the table in its own row order or
+// column order, which depends on the input but not on chance): a stable counting sort of the
+// positions by (prefix, table id, padding).  One CTA per (example, view); integer work only.
 #include "mate_internal.h"
 
 namespace mate {
@@ -8,7 +8,9 @@ namespace mate {
 namespace {
 
 constexpr int kPlanThreads = 1024;
-constexpr int kSmemIds = 4096;  // id histograms up to this many entries live in shared memory
+constexpr int kPlanWarps = kPlanThreads / 32;
+constexpr int kSmemIds = 2048;    // id tables up to this many entries live in shared memory ...
+constexpr int kSmemHist = 8192;   // ... and so do the per-slice tables of the scatter (slices x ids entries)
 
 __device__ __forceinline__ int warp_inclusive_scan(int v, int lane) {
 #pragma unroll
@@ -25,7 +27,8 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
             int group,
             ViewPlan rowv, ViewPlan colv, int32_t *__restrict__ n_valid_out,
             int32_t *__restrict__ status) {
-    __shared__ int32_t s_cursor[kSmemIds];
+    __shared__ int32_t s_tot[kSmemIds];
+    __shared__ int32_t s_hist[kSmemHist];
     __shared__ int s_n_valid;
 
     const int b = blockIdx.x, view = blockIdx.y;
@@ -33,14 +36,23 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
     const ViewPlan &vp = view ? colv : rowv;
     const int32_t *ids = (view ? col_ids : row_ids) + (size_t)b * N;
     const int32_t *oth = (view ? row_ids : col_ids) + (size_t)b * N;
-    const int S = vp.max_id + 2;
+    const int S = vp.max_id + 2;  // one slot per id and one behind them, which counts the padding
     int32_t *seg_off = vp.seg_off + (size_t)b * S;
     int32_t *perm = vp.perm + (size_t)b * N;
     int32_t *inv_perm = vp.inv_perm + (size_t)b * N;
-    volatile int32_t *cur = (S <= kSmemIds) ? s_cursor : (vp.cursor + (size_t)b * S);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    for (int i = tid; i < S; i += kPlanThreads) cur[i] = 0;
+    // The positions are cut into W slices of L consecutive positions (a multiple of 32), one warp
+    // per slice in the scatter; every slice has its own table of S cursors.  With one slice the
+    // table is the id table itself (shared memory, or global memory when there are many ids).
+    const int W = (S <= kSmemIds) ? max(1, min(kPlanWarps, kSmemHist / S)) : 1;
+    const int L = ((N + W - 1) / W + 31) & ~31;
+    volatile int32_t *tot = (S <= kSmemIds) ? s_tot : (vp.cursor + (size_t)b * S);
+    volatile int32_t *hist = (W > 1) ? s_hist : tot;
+
+    for (int i = tid; i < S; i += kPlanThreads) tot[i] = 0;
+    if (W > 1)
+        for (int i = tid; i < W * S; i += kPlanThreads) hist[i] = 0;
     __syncthreads();
 
     // A position is a table token iff it lies behind the prefix and both ids are valid; anything
@@ -51,34 +63,47 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
         return k >= P && id >= 0 && id <= vp.max_id && oth[k] >= 0;
     };
 
-    // 1. validate + histogram of table ids
+    // 1. validate + per-slice histogram of the table ids (padding counts under the last slot)
     bool bad = false;
     for (int k = tid; k < N; k += kPlanThreads) {
         int id = ids[k], o = oth[k];
+        int slot = -1;
         if (k < P) {
             bad |= (id != 0) | (o != 0);
         } else if (id < 0) {
             bad |= (o >= 0);
+            slot = S - 1;
         } else if (o < 0 || id > vp.max_id) {
             bad = true;
+            slot = S - 1;
         } else {
-            atomicAdd((int *)&cur[id], 1);
+            slot = id;
         }
+        if (slot >= 0) atomicAdd((int *)&hist[(k / L) * S + slot], 1);
     }
     if (bad) atomicOr(status, 1);
     __syncthreads();
+    if (W > 1) {
+        for (int i = tid; i < S; i += kPlanThreads) {
+            int sum = 0;
+            for (int w = 0; w < W; ++w) sum += hist[w * S + i];
+            tot[i] = sum;
+        }
+        __syncthreads();
+    }
 
-    // 2. exclusive scan of the histogram -> segment offsets (warp 0, 32 entries per step)
+    // 2. exclusive scan of the id counts -> segment offsets (warp 0, 32 entries per step); the
+    //    padding slot is left out of the sums and so receives the number of valid positions
     if (warp == 0) {
         int carry = P;
         for (int base = 0; base < S; base += 32) {
             int i = base + lane;
-            int c = (i < S - 1) ? cur[i] : 0;
+            int c = (i < S - 1) ? tot[i] : 0;
             int incl = warp_inclusive_scan(c, lane);
             int excl = carry + incl - c;
             if (i < S) {
                 seg_off[i] = excl;
-                cur[i] = excl;
+                tot[i] = excl;
             }
             carry += __shfl_sync(0xffffffffu, incl, 31);
         }
@@ -89,31 +114,40 @@ plan_kernel(const int32_t *__restrict__ row_ids, const int32_t *__restrict__ col
     }
     __syncthreads();
     const int n_valid = s_n_valid;
+    if (W > 1) {  // cursor of (slice, id): the id's offset plus what the slices in front hold of it
+        for (int i = tid; i < S; i += kPlanThreads) {
+            int run = tot[i];
+            for (int w = 0; w < W; ++w) {
+                const int c = hist[w * S + i];
+                hist[w * S + i] = run;
+                run += c;
+            }
+        }
+        __syncthreads();
+    }
 
-    // 3. stable scatter (warp 0 walks the positions in order, 32 at a time; lanes holding the same
-    //    id are ranked by lane, so equal ids keep their original order)
-    if (warp == 0) {
-        int pad_cursor = n_valid;
-        for (int base = 0; base < N; base += 32) {
+    // 3. stable scatter: one warp per slice walks its positions in order, 32 at a time; lanes
+    //    holding the same id are ranked by lane, so equal ids keep their original order
+    if (warp < W) {
+        volatile int32_t *cur = hist + warp * S;
+        const int k_end = min(N, (warp + 1) * L);
+        for (int base = warp * L; base < k_end; base += 32) {
             int k = base + lane;
             bool in = k < N;
             bool table = in && is_table(k);
             bool padding = in && !table && k >= P;
-            int id = table ? ids[k] : 0;
-            int key = table ? id : (padding ? -1 : (int)0x80000000 + lane);
+            int slot = table ? ids[k] : S - 1;
+            bool counted = table || padding;
+            int key = counted ? slot : (int)0x80000000 + lane;
             unsigned grp = __match_any_sync(0xffffffffu, key);
             int rank = __popc(grp & ((1u << lane) - 1u));
             int cnt = __popc(grp);
             int basep = 0;
-            if (table) basep = cur[id];
+            if (counted) basep = cur[slot];
             __syncwarp();
-            if (table && rank == 0) cur[id] = basep + cnt;
+            if (counted && rank == 0) cur[slot] = basep + cnt;
             __syncwarp();
-            int n_pad = __popc(__ballot_sync(0xffffffffu, padding));
-            int pos = k;  // prefix tokens keep their positions
-            if (table) pos = basep + rank;
-            if (padding) pos = pad_cursor + rank;
-            pad_cursor += n_pad;
+            int pos = counted ? basep + rank : k;  // prefix tokens keep their positions
             if (in) {
                 perm[pos] = k;
                 inv_perm[k] = pos;
