@@ -258,7 +258,7 @@ def run_mate(args, cfg):
     torch.cuda.synchronize()
     set_bytes = sum(t.numel() * t.element_size() for t in sets[0].values()) + 3 * sets[0]["Q"].numel() * 2
 
-    fwd_impl = mate.IMPL_AUTO | (mate.FLAG_BULK_TILES if args.loader == "bulk" else 0)
+    fwd_impl = mate.IMPL_AUTO | {"auto": 0, "bulk": mate.FLAG_BULK_TILES, "gather": mate.FLAG_GATHER_TILES}[args.loader]
 
     def step(d):
         mate.mate_attn_fwd(plan, d["Q"], d["K"], d["V"], scale, fwd_impl, out=d["O"], lse=d["LSE"])
@@ -576,9 +576,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--trace", action="store_true",
                     help="print the per-role cycle counters of the profiling build instead of timing")
-    ap.add_argument("--loader", default="gather", choices=["gather", "bulk"],
-                    help="forward K/V tiles that are contiguous in the tensors: row-by-row gathers like every other "
-                         "tile (default) or bulk tensor copies")
+    ap.add_argument("--loader", default="auto", choices=["auto", "gather", "bulk"],
+                    help="forward K/V tiles that are contiguous in the tensors: the library's choice (default: bulk "
+                         "tensor copies from 2048 positions on), row-by-row gathers like every other tile, or bulk "
+                         "tensor copies")
     args = ap.parse_args()
     cfg = tables.CONFIGS[args.workload]
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "mate":

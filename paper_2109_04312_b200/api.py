@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libmate.so")
 
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
-FLAG_VIEW_ORDER, FLAG_BULK_TILES = 4, 8   # or-ed to the implementation choice (see mate.h)
+FLAG_VIEW_ORDER, FLAG_BULK_TILES, FLAG_GATHER_TILES = 4, 8, 16   # or-ed to the implementation choice (see mate.h)
 VIEW_ROW, VIEW_COL = 0, 1
 _BF16, _F32 = 0, 1
 

@@ -590,7 +590,9 @@ static int check_common(const mate_plan_t *plan, int d, int dtype, unsigned flag
     if (dtype != MATE_BF16 && dtype != MATE_F32) return MATE_ERR_UNSUPPORTED;
     if (d <= 0 || d % 8 != 0 || d > 128) return MATE_ERR_UNSUPPORTED;
     const unsigned impl = flags & 3u;
-    if (impl == 3u || (flags & ~(3u | MATE_FLAG_VIEW_ORDER | MATE_FLAG_BULK_TILES))) return MATE_ERR_INVALID_ARG;
+    constexpr unsigned kLoaderBits = MATE_FLAG_BULK_TILES | MATE_FLAG_GATHER_TILES;
+    if (impl == 3u || (flags & ~(3u | MATE_FLAG_VIEW_ORDER | kLoaderBits)) || (flags & kLoaderBits) == kLoaderBits)
+        return MATE_ERR_INVALID_ARG;
     const bool tc_ok = mate::tc_supported(d, dtype);
     if (impl == MATE_IMPL_TCGEN05 && !tc_ok) return MATE_ERR_UNSUPPORTED;
     *use_tc = (impl == MATE_IMPL_TCGEN05) || (impl == MATE_IMPL_AUTO && tc_ok);

@@ -26,10 +26,15 @@ def test_bulk_copies_and_gathers_give_the_same_bits(name, shuffle):
     m, hv, plan = _plan(cfg, rows, cols)
     Q, K, V = (hp.to_dev(vals[n], cfg.dtype) for n in ("Q", "K", "V"))
     O1, L1 = m.mate_attn_fwd(plan, Q, K, V, None, m.IMPL_TCGEN05 | m.FLAG_BULK_TILES)
-    O2, L2 = m.mate_attn_fwd(plan, Q, K, V, None, m.IMPL_TCGEN05)
+    O2, L2 = m.mate_attn_fwd(plan, Q, K, V, None, m.IMPL_TCGEN05 | m.FLAG_GATHER_TILES)
+    O3, L3 = m.mate_attn_fwd(plan, Q, K, V, None, m.IMPL_TCGEN05)   # the library's own choice
     torch.cuda.synchronize()
     plan.status()
     assert torch.equal(O1, O2) and torch.equal(L1, L2)
+    assert torch.equal(O1, O3) and torch.equal(L1, L3)
+    with pytest.raises(m.MateError) as e:   # the two loader bits exclude each other
+        m.mate_attn_fwd(plan, Q, K, V, None, m.IMPL_TCGEN05 | m.FLAG_BULK_TILES | m.FLAG_GATHER_TILES)
+    assert e.value.status == -1
     # and both are the oracle's result (the default path is also covered by the parity tests)
     if name != "long":
         oO, _ = oracle.fwd(vals["Q"], vals["K"], vals["V"], rows, cols, cfg.P, hv, 1.0 / np.sqrt(cfg.d))
