@@ -45,7 +45,6 @@ constexpr int kLoadWarp0 = 10;
 constexpr int kLoadWarps = 2;
 constexpr int kLoadThreads = 32 * kLoadWarps;
 constexpr int kThreads = 32 * (kLoadWarp0 + kLoadWarps);
-constexpr int kBulkFromN = 2048;  // default loader: bulk tensor copies from this sequence length on
 constexpr int kStages = 5;                   // K/V ring
 constexpr int kLag = 2;                      // loader: copy groups in flight behind the newest one
 
@@ -971,12 +970,11 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
     if (g_smem_attr.ensure((const void *)tc_fwd_kernel, (int)kSmemBytes, plan->device) != MATE_OK) return MATE_ERR_CUDA;
     Params p;
     const size_t rows = plan->n_rows();
-    // Bulk tensor copies for the K/V tiles that are contiguous in the caller's tensors: on request, always
-    // for tensors in view order, and by default for long sequences (they measured 2-4 % faster than
-    // row-by-row gathers from 2048 positions on and 7 % slower at 512).  Without the driver entry point
-    // every tile is gathered.
-    const bool want_bulk = (flags & (MATE_FLAG_BULK_TILES | MATE_FLAG_VIEW_ORDER)) ||
-                           (!(flags & MATE_FLAG_GATHER_TILES) && plan->N >= kBulkFromN);
+    // Bulk tensor copies for the K/V tiles that are contiguous in the caller's tensors: on request, and
+    // always for tensors in view order.  Otherwise every tile is gathered row by row (inside whole steps
+    // the two differ by about 1 % either way, depending on the workload), as it is when the driver entry
+    // point for tensor maps is missing.
+    const bool want_bulk = (flags & (MATE_FLAG_BULK_TILES | MATE_FLAG_VIEW_ORDER)) != 0;
     p.use_tma = want_bulk && rows < (size_t(1) << 31) && make_row_map(&p.tmK, K, rows) && make_row_map(&p.tmV, V, rows);
     p.view_order = (flags & MATE_FLAG_VIEW_ORDER) ? 1 : 0;
     p.Q = (const __nv_bfloat16 *)Q;
