@@ -893,6 +893,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_consta
                     commit_and_signal(bar_kv);
                     TR_ADD(3, t_cs);
                 }
+                // The very first tile of the CTA: the other warps are waiting for it, so it (and Q) are
+                // signalled as soon as they have landed, not two tiles later.
+                if (kv_cnt == 0) flush();
                 TR_INC(4);
                 ++kv_cnt;
             }

@@ -16,7 +16,6 @@ constexpr int kUnitRows = 256;   // query rows per unit of the tensor-core kerne
 // what the key range of a table row is made of (plan kernel step 4 and its host twin)
 enum { kBoundsOwn = 0, kBoundsBefore = 1, kBoundsAfter = 2 };
 constexpr int kTraceCtas = 256;  // CTAs whose cycle counters a -DMATE_TRACE build keeps
-constexpr int kTraceEvents = 2048;  // time-stamped events per role of CTA 0 in such a build
 
 // One unit of work of the tensor-core forward: up to 256 consecutive query rows (view order) of one
 // (example, head) -- half 0 = the first 128 rows, half 1 = the rest -- and the key tiles (128 wide)
@@ -191,20 +190,10 @@ int tc_fwd(const mate_plan_t *plan, const void *Q, const void *K, const void *V,
 // the tensor-core kernels, per CTA and role, in a local array `tr`.  Profiling aid only; compiled
 // out of the library.
 #ifdef MATE_TRACE
-// event log of CTA 0 (two roles, time-stamped): TR_EV(role, id) in one lane of a warp
-#define TR_EV(role, id)                                                              \
-    do {                                                                             \
-        if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && ev_n < mate::kTraceEvents) { \
-            mate::g_evlog[((role) * mate::kTraceEvents + ev_n) * 2] = (id);            \
-            mate::g_evlog[((role) * mate::kTraceEvents + ev_n) * 2 + 1] = clock64();   \
-            ++ev_n;                                                                  \
-        }                                                                            \
-    } while (0)
 #define TR_T0(var) const long long var = clock64()
 #define TR_ADD(cat, var) tr[cat] += clock64() - (var)
 #define TR_INC(cat) tr[cat] += 1
 #else
-#define TR_EV(role, id)
 #define TR_T0(var)
 #define TR_ADD(cat, var)
 #define TR_INC(cat)
