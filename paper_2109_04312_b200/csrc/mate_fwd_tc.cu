@@ -402,6 +402,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_fwd_kernel(const __grid_consta
 
                 bool two_pass = first;
                 TR_T0(t_p2);
+                if (first) {
+                    // A unit's first tile has no running max yet.  The max over the first 32 columns in which
+                    // the warp has keys serves as the base when every row of the warp has a key there: the
+                    // one-pass path below then runs as for any other tile (and still falls back to two passes
+                    // when a row's max over the whole tile lies more than the threshold above that base).
+                    const int cq = max(ch0, e_lo_min > 0 ? e_lo_min >> 5 : 0);
+                    if (cq < ch1 && cq * 32 < e_hi_max) {
+                        float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                        uint32_t v[32];
+                        tmem_ld32(tS + cq * 32, v);
+                        tc_wait_ld();
+                        if (!(cq * 32 >= e_lo_max && cq * 32 + 32 <= e_hi_min)) chunk_mask(v, cq * 32, r_lo, r_span);
+                        chunk_max(v, tm);
+                        const float t = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3])) * p.scale_log2;
+                        if (__all_sync(0xffffffffu, t > -INFINITY)) {
+                            m2 = t;
+                            two_pass = false;
+                        }
+                    }
+                }
                 if (!two_pass) {
                     // one pass with the running max; the tile's own max is known before S is given up
                     float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
