@@ -577,8 +577,8 @@ def main():
     ap.add_argument("--trace", action="store_true",
                     help="print the per-role cycle counters of the profiling build instead of timing")
     ap.add_argument("--loader", default="auto", choices=["auto", "gather", "bulk"],
-                    help="forward K/V tiles that are contiguous in the tensors: the library's default (gathers), "
-                         "row-by-row gathers stated explicitly, or bulk tensor copies")
+                    help="forward K/V tiles that are contiguous in the tensors: the library's default (bulk tensor "
+                         "copies), row-by-row gathers like every other tile, or bulk tensor copies stated explicitly")
     args = ap.parse_args()
     cfg = tables.CONFIGS[args.workload]
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "mate":

@@ -71,11 +71,11 @@ enum { MATE_IMPL_AUTO = 0, MATE_IMPL_SIMT = 1, MATE_IMPL_TCGEN05 = 2 };
  *   BULK_TILES   the tensor-core forward fetches the K/V tiles that are contiguous in the tensors -- the
  *                prefix block of every head and, for a row-major table, every tile of the row view --
  *                with bulk tensor copies (one per tile and matrix) instead of row-by-row gathers.  Same
- *                results bit for bit.
- *   GATHER_TILES every K/V tile is gathered row by row: the default, so the bit only states it.
- *                (Timed inside whole forward + backward steps on sequences of 512 to 8192 positions,
- *                bulk copies gain about 1 % on two workloads and lose up to 1.5 % on the other two.)
- *                Both bits together: MATE_ERR_INVALID_ARG. */
+ *                results bit for bit.  This is the default wherever the driver provides tensor maps,
+ *                so the bit only states it.
+ *   GATHER_TILES every K/V tile is gathered row by row.  (Timed back to back on sequences of 512 to
+ *                8192 positions, bulk copies are 2-3 % faster on two workloads, equal on one and
+ *                0.6 % slower on one.)  Both bits together: MATE_ERR_INVALID_ARG. */
 enum { MATE_FLAG_VIEW_ORDER = 4, MATE_FLAG_BULK_TILES = 8, MATE_FLAG_GATHER_TILES = 16 };
 
 const char *mate_status_string(int status);
