@@ -7,13 +7,15 @@
 //   warps 4-7   softmax of half 1 (rows 128..255)
 //   warps 8, 9  one thread each issues the tcgen05.mma of half 0 / half 1
 //   warps 10-11 loaders: gather Q, K, V rows by view-order index into 128-byte swizzled shared
-//               memory with 16-byte cp.async (the gather of Section 3.1 fused into the loads)
+//               memory with 16-byte cp.async (the gather of Section 3.1 fused into the loads); K/V
+//               tiles whose rows lie in place in the tensors come in by one bulk tensor copy each
 //
 // Per key tile and half:   S = Q K^T  (tcgen05.mma, M = 128, N <= 128, K = 64, accumulator in TMEM)
-//                          online softmax in the exp2 domain: P = exp2(S c - m), row sum.  After a
-//                          unit's first tile, P is formed in one pass over S with the running max m;
-//                          the tile's own max is tracked on the way and only a growth by more than
-//                          2^8 sends the tile through the two-pass path (max, rescale O, exp)
+//                          online softmax in the exp2 domain: P = exp2(S c - m), row sum.  P is
+//                          formed in one pass over S with the running max m (for a unit's first
+//                          tile: the max over its first 32 columns); the tile's own max is tracked
+//                          on the way and only a growth by more than 2^8 sends the tile through
+//                          the two-pass path (max, rescale O, exp)
 //                          O += P V   (tcgen05.mma, M = 128, N = 64, P read from TMEM; O stays there)
 // S is released to the MMA issuer as soon as its last 32 columns sit in registers, so the Q K^T of
 // the half's next tile runs under the rest of the exponentials.
