@@ -148,9 +148,8 @@ def test_packed_equals_padded():
             L = cu[b + 1] - cu[b]
             assert torch.equal(Oa[:, cu[b]:cu[b + 1]], Op[b, :, :L])
             assert torch.equal(La[:, cu[b]:cu[b + 1]], Lp[b, :, :L])
-            if impl == m.IMPL_SIMT:   # the tensor-core backward adds dK / dV with atomics: order may differ
-                for x, y in zip(ga, gp):
-                    assert torch.equal(x[:, cu[b]:cu[b + 1]], y[b, :, :L])
+            for x, y in zip(ga, gp):   # no gradient is accumulated across CTAs: the same bits here too
+                assert torch.equal(x[:, cu[b]:cu[b + 1]], y[b, :, :L])
     packed.status()
     padded.status()
     packed.destroy()
